@@ -1,0 +1,230 @@
+/*
+ * cascade_ffn.h -- C ABI of the streamFFN routed-expert path for one B200 (sm_100a).
+ *
+ * The library runs the expert side of a prefill MoE layer the way the paper's
+ * streamFFN does (Section 3.2 "Asynchronous EP and streaming FFN"; Appendix
+ * "Runtime Implementation Details"): routed tokens arrive in per-replica chunks at
+ * different times; ready chunks accumulate until a launch threshold theta is reached
+ * (or everything has arrived: the final flush bypasses theta); every launch is one
+ * *grouped FFN invocation* on its own CUDA stream and scratch slot:
+ *
+ *   layout transform  histogram -> exclusive scan -> stable scatter into expert-major,
+ *                     tile-aligned groups, with an inverse map (Appendix "Grouped FFN
+ *                     invocations")
+ *   expert GEMM 1     [gate | up] projections, SiLU(gate)*up fused in the epilogue
+ *   expert GEMM 2     down projection
+ *   combine           every routed contribution weighted by its routing coefficient
+ *                     exactly once, accumulated per token, written in token order
+ *                     (Appendix "Output return and combine")
+ *
+ * Conventions
+ *   - Every function returns 0 (CEP_OK) or a negative cep_status.  Nothing throws,
+ *     aborts or traps.  cep_last_error() gives a human-readable reason.
+ *   - Pointers marked [device] are CUDA device pointers, [host] are host pointers.
+ *   - The CALLER owns every device buffer (workspace, packed weights, chunk inputs,
+ *     output).  The library allocates no device memory; it owns only the host-side
+ *     plan object and the CUDA streams/events it creates.
+ *   - Chunk input buffers and the output buffer must stay valid and unmodified from
+ *     ffn_submit_chunk() until the stream passed to combine() has completed: buffers
+ *     remain live until their dependent computations have finished (Appendix "Output
+ *     return and combine").
+ *   - ffn_submit_chunk / ffn_flush / combine only enqueue work; none blocks the host
+ *     on the device.
+ *   - A plan is not thread-safe; use one plan per host thread or serialise calls.
+ *   - Expert ids are *global*; ids 0..n_experts_local-1 live on this rank, larger ids
+ *     belong to other ranks and their pairs are skipped.
+ */
+#ifndef CASCADE_FFN_H_
+#define CASCADE_FFN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CEP_API __attribute__((visibility("default")))
+#else
+#define CEP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cep_plan cep_plan;
+
+typedef enum {
+  CEP_OK = 0,
+  CEP_ERR_ARG = -1,            /* null pointer, non-positive size, unsupported shape            */
+  CEP_ERR_STATE = -2,          /* call out of order: submit before begin / after flush, double
+                                  submit of a chunk id, begin while a layer is open             */
+  CEP_ERR_WORKSPACE = -3,      /* workspace or packed-weight buffer too small or misaligned     */
+  CEP_ERR_CAPACITY = -4,       /* more tokens or chunks than the plan was made for              */
+  CEP_ERR_INCOMPLETE = -5,     /* flush/combine with fewer chunks than ffn_begin announced;
+                                  the work already submitted still runs                          */
+  CEP_ERR_BAD_ROUTING = -6,    /* device found an expert id outside [0, n_experts_global)       */
+  CEP_ERR_DEVICE_TIMEOUT = -7, /* a bounded wait inside a kernel expired; kernel exited cleanly */
+  CEP_ERR_CUDA = -8,           /* a CUDA runtime/driver call failed                             */
+  CEP_ERR_UNSUPPORTED = -9     /* valid request this build does not implement                   */
+} cep_status;
+
+typedef enum {
+  CEP_BF16 = 0,                /* bf16 activations and weights, fp32 accumulate, bf16 output    */
+  CEP_FP8_E4M3_BLOCK128 = 1    /* e4m3 codes; fp32 scales per 1x128 activation block and per
+                                  128x128 weight block; bf16 output                              */
+} cep_dtype;
+
+/* Execution modes of the ablation in Section 5.4. */
+typedef enum {
+  CEP_MODE_SYNC = 0,           /* one invocation once all chunks have arrived                   */
+  CEP_MODE_ASYNC = 1,          /* one invocation per chunk as it arrives                        */
+  CEP_MODE_STREAMFFN = 2       /* accumulate to threshold_pairs, multi-stream, final flush      */
+} cep_mode;
+
+typedef enum {
+  CEP_GEMM_TCGEN05 = 0,        /* tcgen05/TMEM tiles fed by TMA (the product path)              */
+  CEP_GEMM_SIMT = 1            /* slow CUDA-core kernel, kept for fault isolation in tests      */
+} cep_gemm_impl;
+
+#define CEP_MAX_CHUNKS_PER_INVOCATION 32   /* a batch is launched early when it holds this many */
+#define CEP_ROW_ALIGN 128                  /* expert groups start on multiples of the GEMM tile */
+
+typedef struct {
+  int32_t hidden;              /* H; multiple of 128 (bf16: multiple of 64)                     */
+  int32_t inter;               /* I; multiple of 128                                            */
+  int32_t n_experts_global;    /* E_g                                                           */
+  int32_t n_experts_local;     /* E <= E_g, at most 1024                                        */
+  int32_t top_k;               /* k, at most 32                                                 */
+  int32_t max_tokens;          /* upper bound on tokens per layer call                          */
+  int32_t max_chunks;          /* upper bound on chunks per layer call                          */
+  int32_t dtype;               /* cep_dtype                                                     */
+  int32_t mode;                /* cep_mode                                                      */
+  int32_t n_streams;           /* S >= 1 compute streams / scratch slots (round-robin)          */
+  int64_t threshold_pairs;     /* theta: ready local (token, expert) pairs per invocation       */
+  int32_t gemm_impl;           /* cep_gemm_impl                                                 */
+  int32_t debug_checks;        /* nonzero: kernels bounds-check every index and record, never
+                                  trap, on violation                                            */
+} cep_config;
+
+/* Per-invocation record for tracing (ffn_query). */
+typedef struct {
+  int32_t n_chunks;            /* chunks in the batch                                           */
+  int32_t first_chunk_pos;     /* submission position of its first chunk                        */
+  int32_t stream_index;        /* compute stream / scratch slot used                            */
+  int32_t n_tokens;            /* tokens in the batch                                           */
+  int64_t pairs_bound;         /* host-side count of ready pairs that triggered the launch      */
+  float elapsed_ms;            /* device time first kernel -> last kernel; < 0 if not finished  */
+} cep_invocation_info;
+
+/* Bytes of device workspace a plan with this configuration needs.  [host] out. */
+CEP_API int moe_plan_workspace_bytes(const cep_config* cfg, size_t* bytes);
+
+/* Bytes of the packed (K-major, gate/up interleaved) copy of the expert weights. */
+CEP_API int moe_packed_weight_bytes(const cep_config* cfg, size_t* bytes);
+
+/*
+ * moe_plan: create a plan ("routing" = the shapes and the streamFFN policy of one MoE
+ * layer).  `workspace` [device], 256-byte aligned, at least moe_plan_workspace_bytes();
+ * it is carved into S scratch slots (each invocation has its own scratch, Appendix
+ * "Grouped FFN invocations") and stays owned by the caller.  Creates S non-blocking
+ * streams and the events.  Must be called with the target device current.
+ */
+CEP_API int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep_plan** out);
+
+/*
+ * One-off weight prepack, off the hot path.  Inputs [device]:
+ *   w_gate, w_up  [E, H, I]   w_down [E, I, H]     (bf16, or e4m3 codes)
+ *   s_gate, s_up  [E, H/128, I/128]  s_down [E, I/128, H/128]   fp32, fp8 only, else NULL
+ * `packed` [device], 256-byte aligned, moe_packed_weight_bytes() long, must outlive the
+ * plan's use of it.  The transposes are enqueued on `stream` (cudaStream_t); later
+ * layer calls are ordered after them.
+ */
+CEP_API int moe_load_weights(cep_plan* plan, const void* w_gate, const void* w_up, const void* w_down,
+                     const float* s_gate, const float* s_up, const float* s_down,
+                     void* packed, size_t packed_bytes, void* stream);
+
+/*
+ * Open a layer call.  `out` [device] bf16 [n_tokens_total, H] in token order; every row
+ * is written by combine work (rows of tokens with no local expert become exact zeros).
+ * n_chunks_expected chunks will be submitted, together covering the n_tokens_total
+ * tokens exactly once.
+ */
+CEP_API int ffn_begin(cep_plan* plan, void* out, int32_t n_tokens_total, int32_t n_chunks_expected);
+
+/*
+ * A replica's routed tokens have arrived (Section 3.2: per-replica completion signal).
+ *   chunk_id       0..n_chunks_expected-1, each exactly once, any order
+ *   token_offset   first token (row of `out`) this chunk covers
+ *   tokens         [device] bf16 [n,H]  |  e4m3 [n,H]
+ *   token_scales   [device] fp32 [n,H/128] for fp8, else NULL
+ *   topk_ids       [device] int32 [n,k] global expert ids, distinct per token
+ *   topk_weights   [device] fp32 [n,k]
+ *   n_local_pairs  number of (token,slot) pairs with id < n_experts_local, as known from
+ *                  dispatch metadata; -1 => use the bound n*k.  Only the launch decision
+ *                  uses it, never an index.
+ *   stream         cudaStream_t on which the chunk's data becomes ready; the library
+ *                  records an event there and its compute streams wait on it.
+ * Returns immediately.  May launch an invocation (see cep_mode).
+ */
+CEP_API int ffn_submit_chunk(cep_plan* plan, int32_t chunk_id, int32_t token_offset, int32_t n_tokens,
+                     const void* tokens, const float* token_scales, const int32_t* topk_ids,
+                     const float* topk_weights, int64_t n_local_pairs, void* stream);
+
+/* All tokens have arrived: launch whatever is pending regardless of theta
+ * (Section 3.2 "Launch threshold", last sentence). */
+CEP_API int ffn_flush(cep_plan* plan);
+
+/*
+ * Layer boundary (Appendix "Output return and combine": the common layer boundary is
+ * retained).  Makes `stream` wait for every invocation of this layer call, then
+ * enqueues the read-back of the device status word.  `out` is complete once `stream`
+ * has completed.  Implies ffn_flush.  Closes the layer call.
+ */
+CEP_API int combine(cep_plan* plan, void* stream);
+
+/* Device-side status of the last closed layer call.  Valid after the stream given to
+ * combine() has completed (the caller synchronises); before that returns CEP_ERR_STATE.
+ * CEP_OK, CEP_ERR_BAD_ROUTING or CEP_ERR_DEVICE_TIMEOUT. */
+CEP_API int ffn_status(cep_plan* plan);
+
+/* Number of invocations launched in the current / last layer call. */
+CEP_API int ffn_num_invocations(const cep_plan* plan);
+
+/* Trace record of invocation `inv` [host out]. elapsed_ms needs the invocation finished. */
+CEP_API int ffn_query(cep_plan* plan, int32_t inv, cep_invocation_info* info);
+
+/*
+ * Copy the layout transform's integers of invocation `inv` to [host] arrays (any may be
+ * NULL): counts[E], offsets[E+1], padded_offsets[E+1], row_of_pair[n_tokens*k] (physical,
+ * tile-aligned row of each pair in batch pair order, -1 if not local), pair_of_row[
+ * padded_offsets[E]] (inverse, -1 on padding rows).  Synchronises the invocation's stream.
+ * Only meaningful until the invocation's scratch slot is reused (S invocations later).
+ */
+CEP_API int ffn_debug_export(cep_plan* plan, int32_t inv, int32_t* counts, int32_t* offsets,
+                     int32_t* padded_offsets, int32_t* row_of_pair, int32_t* pair_of_row);
+
+/* Total kernel launches this plan has issued (layout, GEMM, combine, prepack). */
+CEP_API int64_t cep_kernel_launches(const cep_plan* plan);
+
+/* Destroys streams, events and the host object.  Synchronises the plan's streams. */
+CEP_API int moe_plan_destroy(cep_plan* plan);
+
+/* Static or plan-owned string describing the last error on this plan (or the last
+ * plan-less error when plan is NULL). */
+CEP_API const char* cep_last_error(const cep_plan* plan);
+
+/*
+ * Host-only helpers exported for CPU tests of the index arithmetic the kernels use.
+ * cep_debug_decode_tile: maps a linear tile index to (expert, m_block, n_block) given the
+ * per-expert m-tile prefix [E+1] and the number of n blocks; returns 0 or CEP_ERR_ARG.
+ * cep_debug_schedule: replays the host scheduler on a list of per-chunk pair counts and
+ * writes, per chunk position, the invocation it lands in; returns the invocation count.
+ */
+CEP_API int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n,
+                          int32_t tile, int32_t* expert, int32_t* m_block, int32_t* n_block);
+CEP_API int cep_debug_schedule(const int64_t* pairs, int32_t n_chunks, int32_t mode, int64_t theta,
+                       int32_t* invocation_of_chunk);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASCADE_FFN_H_ */

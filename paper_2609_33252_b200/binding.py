@@ -1,0 +1,274 @@
+"""ctypes binding of include/cascade_ffn.h: same names, argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels.  torch is used for
+device memory and streams.  If the library cannot be loaded the import of a symbol
+raises: there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libcascade_ffn.so")
+
+CEP_BF16, CEP_FP8_E4M3_BLOCK128 = 0, 1
+CEP_MODE_SYNC, CEP_MODE_ASYNC, CEP_MODE_STREAMFFN = 0, 1, 2
+CEP_GEMM_TCGEN05, CEP_GEMM_SIMT = 0, 1
+STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ERR_WORKSPACE",
+                -4: "CEP_ERR_CAPACITY", -5: "CEP_ERR_INCOMPLETE", -6: "CEP_ERR_BAD_ROUTING",
+                -7: "CEP_ERR_DEVICE_TIMEOUT", -8: "CEP_ERR_CUDA", -9: "CEP_ERR_UNSUPPORTED"}
+
+EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
+           "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
+           "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
+           "cep_debug_decode_tile", "cep_debug_schedule"]
+
+
+class CepConfig(ctypes.Structure):
+    _fields_ = [("hidden", ctypes.c_int32), ("inter", ctypes.c_int32),
+                ("n_experts_global", ctypes.c_int32), ("n_experts_local", ctypes.c_int32),
+                ("top_k", ctypes.c_int32), ("max_tokens", ctypes.c_int32), ("max_chunks", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("n_streams", ctypes.c_int32),
+                ("threshold_pairs", ctypes.c_int64), ("gemm_impl", ctypes.c_int32),
+                ("debug_checks", ctypes.c_int32)]
+
+
+class InvocationInfo(ctypes.Structure):
+    _fields_ = [("n_chunks", ctypes.c_int32), ("first_chunk_pos", ctypes.c_int32),
+                ("stream_index", ctypes.c_int32), ("n_tokens", ctypes.c_int32),
+                ("pairs_bound", ctypes.c_int64), ("elapsed_ms", ctypes.c_float)]
+
+
+class CepError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("%s: %s" % (STATUS_NAMES.get(code, str(code)), msg))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(build_if_missing: bool = True):
+    """dlopen the C-ABI library (building it with nvcc first if it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        from .build import build
+        try:
+            build()
+        except Exception:
+            if not os.path.exists(LIB_PATH):
+                raise
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libcascade_ffn.so is missing: build it with `python -m paper_2609_33252_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    cfgp = ctypes.POINTER(CepConfig)
+    sig = {
+        "moe_plan_workspace_bytes": (ctypes.c_int, [cfgp, ctypes.POINTER(sz)]),
+        "moe_packed_weight_bytes": (ctypes.c_int, [cfgp, ctypes.POINTER(sz)]),
+        "moe_plan": (ctypes.c_int, [cfgp, vp, sz, ctypes.POINTER(vp)]),
+        "moe_load_weights": (ctypes.c_int, [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]),
+        "ffn_begin": (ctypes.c_int, [vp, vp, i32, i32]),
+        "ffn_submit_chunk": (ctypes.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, i64, vp]),
+        "ffn_flush": (ctypes.c_int, [vp]),
+        "combine": (ctypes.c_int, [vp, vp]),
+        "ffn_status": (ctypes.c_int, [vp]),
+        "ffn_num_invocations": (ctypes.c_int, [vp]),
+        "ffn_query": (ctypes.c_int, [vp, i32, ctypes.POINTER(InvocationInfo)]),
+        "ffn_debug_export": (ctypes.c_int, [vp, i32, vp, vp, vp, vp, vp]),
+        "cep_kernel_launches": (i64, [vp]),
+        "moe_plan_destroy": (ctypes.c_int, [vp]),
+        "cep_last_error": (ctypes.c_char_p, [vp]),
+        "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
+        "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = L
+    return L
+
+
+def lib():
+    return load_library()
+
+
+def _check(rc: int, plan=None, allow: Sequence[int] = ()):
+    if rc != 0 and rc not in allow:
+        msg = lib().cep_last_error(plan)
+        raise CepError(rc, msg.decode() if msg else "")
+    return rc
+
+
+def _dptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+# ---------------------------------------------------------------- same-named wrappers
+def moe_plan_workspace_bytes(cfg: CepConfig) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().moe_plan_workspace_bytes(ctypes.byref(cfg), ctypes.byref(n)))
+    return n.value
+
+
+def moe_packed_weight_bytes(cfg: CepConfig) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().moe_packed_weight_bytes(ctypes.byref(cfg), ctypes.byref(n)))
+    return n.value
+
+
+def moe_plan(cfg: CepConfig, workspace) -> int:
+    """workspace: torch uint8 CUDA tensor.  Returns the plan handle."""
+    h = ctypes.c_void_p()
+    _check(lib().moe_plan(ctypes.byref(cfg), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                          ctypes.byref(h)))
+    return h.value
+
+
+def moe_load_weights(plan, w_gate, w_up, w_down, s_gate, s_up, s_down, packed, stream=None):
+    _check(lib().moe_load_weights(plan, _dptr(w_gate), _dptr(w_up), _dptr(w_down), _dptr(s_gate), _dptr(s_up),
+                                  _dptr(s_down), packed.data_ptr(), packed.numel() * packed.element_size(),
+                                  _stream_handle(stream)), plan)
+
+
+def ffn_begin(plan, out, n_tokens_total: int, n_chunks_expected: int):
+    _check(lib().ffn_begin(plan, out.data_ptr(), n_tokens_total, n_chunks_expected), plan)
+
+
+def ffn_submit_chunk(plan, chunk_id: int, token_offset: int, n_tokens: int, tokens, token_scales, topk_ids,
+                     topk_weights, n_local_pairs: int = -1, stream=None):
+    _check(lib().ffn_submit_chunk(plan, chunk_id, token_offset, n_tokens, _dptr(tokens), _dptr(token_scales),
+                                  _dptr(topk_ids), _dptr(topk_weights), n_local_pairs, _stream_handle(stream)),
+           plan)
+
+
+def ffn_flush(plan, allow_incomplete: bool = False) -> int:
+    return _check(lib().ffn_flush(plan), plan, allow=(-5,) if allow_incomplete else ())
+
+
+def combine(plan, stream=None, allow_incomplete: bool = False) -> int:
+    return _check(lib().combine(plan, _stream_handle(stream)), plan, allow=(-5,) if allow_incomplete else ())
+
+
+def ffn_status(plan) -> int:
+    return lib().ffn_status(plan)
+
+
+def ffn_num_invocations(plan) -> int:
+    return lib().ffn_num_invocations(plan)
+
+
+def ffn_query(plan, inv: int) -> InvocationInfo:
+    info = InvocationInfo()
+    _check(lib().ffn_query(plan, inv, ctypes.byref(info)), plan)
+    return info
+
+
+def ffn_debug_export(plan, inv: int, n_experts_local: int, n_pairs: int):
+    """Returns dict of numpy int32 arrays: counts, offsets, padded_offsets, row_of_pair, pair_of_row."""
+    import numpy as np
+    E = n_experts_local
+    counts = np.zeros(E, np.int32)
+    offsets = np.zeros(E + 1, np.int32)
+    padded = np.zeros(E + 1, np.int32)
+    rop = np.full(max(n_pairs, 1), -1, np.int32)
+    p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().ffn_debug_export(plan, inv, p(counts), p(offsets), p(padded), p(rop), None), plan)
+    por = np.full(max(int(padded[E]), 1), -1, np.int32)
+    _check(lib().ffn_debug_export(plan, inv, None, None, None, None, p(por)), plan)
+    return dict(counts=counts, offsets=offsets, padded_offsets=padded, row_of_pair=rop[:n_pairs],
+                pair_of_row=por[:int(padded[E])])
+
+
+def cep_kernel_launches(plan) -> int:
+    return lib().cep_kernel_launches(plan)
+
+
+def moe_plan_destroy(plan):
+    _check(lib().moe_plan_destroy(plan))
+
+
+def cep_last_error(plan=None) -> str:
+    m = lib().cep_last_error(plan)
+    return m.decode() if m else ""
+
+
+def cep_debug_decode_tile(tile_prefix, n_blocks_n: int, tile: int):
+    import numpy as np
+    tp = np.ascontiguousarray(tile_prefix, dtype=np.int32)
+    e, m, n = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    rc = lib().cep_debug_decode_tile(tp.ctypes.data_as(ctypes.c_void_p), tp.shape[0] - 1, n_blocks_n, tile,
+                                     ctypes.byref(e), ctypes.byref(m), ctypes.byref(n))
+    return None if rc else (e.value, m.value, n.value)
+
+
+def cep_debug_schedule(pairs: Sequence[int], mode: int, theta: int) -> List[int]:
+    import numpy as np
+    pr = np.ascontiguousarray(pairs, dtype=np.int64)
+    out = np.zeros(max(len(pr), 1), np.int32)
+    n = lib().cep_debug_schedule(pr.ctypes.data_as(ctypes.c_void_p), len(pr), mode, theta,
+                                 out.ctypes.data_as(ctypes.c_void_p))
+    if n < 0:
+        raise CepError(n, "cep_debug_schedule")
+    return out[:len(pr)].tolist()
+
+
+# ---------------------------------------------------------------- convenience owner of the buffers
+class MoELayer:
+    """Owns the torch-allocated workspace and packed weights of one plan.
+
+    Plumbing only: allocation and pointer passing.  ``run`` submits the chunks of one
+    layer call in the given order on the given streams and joins on ``stream``.
+    """
+
+    def __init__(self, hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
+                 dtype=CEP_BF16, mode=CEP_MODE_STREAMFFN, n_streams=2, threshold_pairs=0,
+                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, device="cuda"):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the streamFFN library needs a CUDA device; there is no CPU path")
+        self.cfg = CepConfig(hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
+                             dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks)
+        self.device = torch.device(device)
+        self.workspace = torch.empty(moe_plan_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
+        self.packed = torch.empty(moe_packed_weight_bytes(self.cfg), dtype=torch.uint8, device=self.device)
+        self.plan = moe_plan(self.cfg, self.workspace)
+
+    def load_weights(self, w_gate, w_up, w_down, s_gate=None, s_up=None, s_down=None, stream=None):
+        moe_load_weights(self.plan, w_gate, w_up, w_down, s_gate, s_up, s_down, self.packed, stream)
+
+    def run(self, out, chunks, order=None, streams=None, stream=None, n_local_pairs=None):
+        """chunks: list of (token_offset, x, x_scale, ids, w).  Returns the number of invocations."""
+        n_tok = sum(c[1].shape[0] for c in chunks)
+        ffn_begin(self.plan, out, n_tok, len(chunks))
+        order = list(range(len(chunks))) if order is None else order
+        for c in order:
+            off, x, xs, ids, w = chunks[c]
+            ffn_submit_chunk(self.plan, c, off, x.shape[0], x, xs, ids, w,
+                             -1 if n_local_pairs is None else n_local_pairs[c],
+                             None if streams is None else streams[c])
+        ffn_flush(self.plan)
+        combine(self.plan, stream)
+        return ffn_num_invocations(self.plan)
+
+    def close(self):
+        if getattr(self, "plan", None):
+            moe_plan_destroy(self.plan)
+            self.plan = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,100 @@
+// Shared declarations of the streamFFN library's translation units (host + device).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/cascade_ffn.h"
+
+namespace cep {
+
+constexpr int kRowAlign = CEP_ROW_ALIGN;        // rows per GEMM M tile; expert groups start on multiples
+constexpr int kMaxChunksPerInv = CEP_MAX_CHUNKS_PER_INVOCATION;
+constexpr int kSegPairs = 2048;                 // pairs per block in the histogram / rank kernels
+constexpr int kGroupM = 16;                     // m-tiles per scheduling group (L2 reuse of A rows)
+constexpr int kQuantBlock = 128;                // fp8 scale block
+
+// Device status word layout (int32 each).
+enum StatusWord { kStBadRouting = 0, kStTimeout = 1, kStBoundsViolation = 2, kStDetail = 3, kStWords = 8 };
+
+// One chunk of a batch as the kernels see it.
+struct ChunkDesc {
+  const void* tokens;         // [n,H] bf16 | e4m3
+  const float* scales;        // fp8: [n,H/128]
+  const int32_t* ids;         // [n,k]
+  const float* weights;       // [n,k]
+  int32_t n_tokens;
+  int32_t token_offset;       // row of `out` of the chunk's first token
+  int32_t token_base;         // index of the chunk's first token inside the batch
+  int32_t pad_;
+};
+
+struct BatchDesc {
+  ChunkDesc chunk[kMaxChunksPerInv];
+  int32_t n_chunks;
+  int32_t n_tokens;           // tokens in the batch
+};
+
+// Per-slot integer scratch produced by the layout transform.
+struct LayoutPtrs {
+  int32_t* counts;            // [E]
+  int32_t* offsets;           // [E+1]
+  int32_t* padded_offsets;    // [E+1]
+  int32_t* tile_prefix;       // [E+1] cumulative number of 128-row tiles
+  int32_t* block_base;        // [n_seg_max, E] per (segment, expert): first histogram, then row base
+  int32_t* row_of_pair;       // [max_tokens*k] physical row, -1 when not local
+  int32_t* pair_of_row;       // [cap_rows] batch pair index, -1 on padding
+  int32_t* status;            // [kStWords]
+};
+
+// ---------------------------------------------------------------- tile scheduling arithmetic
+// Linear tile index -> (expert, m_block, n_block).  Tiles are expert-major; inside an
+// expert, m-tiles are taken in groups of kGroupM, and inside a group the n block is the
+// slow index, so that concurrently running CTAs share one weight tile and a group's
+// activation rows stay L2-resident while the expert's weights stream past them.
+struct TileCoord { int expert, m_block, n_block; };
+
+__host__ __device__ inline bool decode_tile(const int32_t* __restrict__ tile_prefix, int n_experts,
+                                            int n_blocks_n, int tile, TileCoord* out) {
+  if (tile < 0 || n_blocks_n <= 0) return false;
+  int lo = 0, hi = n_experts;            // find e: prefix[e]*NB <= tile < prefix[e+1]*NB
+  if ((long long)tile >= (long long)tile_prefix[n_experts] * n_blocks_n) return false;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if ((long long)tile_prefix[mid] * n_blocks_n <= tile) lo = mid; else hi = mid;
+  }
+  // now prefix[lo] <= tile / NB < prefix[lo+1]: expert lo has tiles and owns this one
+  const int mt = tile_prefix[lo + 1] - tile_prefix[lo];
+  const int li = tile - tile_prefix[lo] * n_blocks_n;
+  const int per_group = kGroupM * n_blocks_n;
+  const int g = li / per_group;
+  const int rem = li - g * per_group;
+  int gm = mt - g * kGroupM;
+  if (gm > kGroupM) gm = kGroupM;
+  out->expert = lo;
+  out->n_block = rem / gm;
+  out->m_block = g * kGroupM + rem % gm;
+  return true;
+}
+
+// ---------------------------------------------------------------- kernel launchers (defined in the .cu files)
+struct GemmProblem {
+  // A operand: rows x K, K contiguous (the permuted activations or the intermediate)
+  // B operand: per expert N x K, K contiguous (packed weights)
+  int K, N;                   // N = columns of the weight panel (2I for GEMM1, H for GEMM2)
+  int n_experts;
+  int swiglu;                 // 1: output column j = silu(acc[:, pair(j)]) * acc[:, pair(j)+128]
+  int out_ld;                 // elements per output row
+  int cap_rows;               // rows the A / output buffers hold
+  int is_fp8;
+};
+
+cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
+                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, int64_t* launches);
+cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp,
+                           const void* y, void* out, cudaStream_t s, int64_t* launches);
+cudaError_t launch_gemm_simt(const GemmProblem& p, const void* a, const void* b, void* out,
+                             const LayoutPtrs& lp, cudaStream_t s, int64_t* launches);
+cudaError_t launch_prepack(const cep_config& cfg, const void* w_gate, const void* w_up, const void* w_down,
+                           void* w13p, void* w2p, cudaStream_t s, int64_t* launches);
+
+}  // namespace cep

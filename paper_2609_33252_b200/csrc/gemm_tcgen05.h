@@ -1,0 +1,22 @@
+// Host interface of the tensor-core grouped GEMM (gemm_tcgen05.cu).
+#pragma once
+#include "cep_common.h"
+
+namespace cep {
+
+// Opaque 128-byte TMA descriptor (layout of the driver's CUtensorMap).
+struct alignas(64) GemmTensorMap { unsigned long long opaque[16]; };
+
+// Describes a K-major operand `rows x K` (n_batch == 0) or `n_batch x rows x K` (n_batch > 0)
+// for 128-byte-of-K x box_rows tiles with 128-byte swizzle.  Returns 0, -1 when the driver
+// entry point is unavailable, -2 when the driver rejects the description.
+int make_operand_map(GemmTensorMap* out, const void* base, int elt_bytes, int K, long long rows, int n_batch,
+                     int box_rows);
+int gemm_tile_rows();
+int gemm_tile_cols();
+
+cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                                void* out, const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s,
+                                int64_t* launches);
+
+}  // namespace cep

@@ -1,0 +1,220 @@
+// Layout transform of one grouped FFN invocation (Appendix "Grouped FFN invocations"):
+// selected rows of the ready chunks are gathered into contiguous, tile-aligned groups by
+// expert, with per-expert offsets computed from the counts and an inverse map kept for
+// the combine.  Four kernels: histogram -> exclusive scan -> stable rank -> row scatter.
+//
+// Pair order inside a batch is (chunk position, token, slot) lexicographic; the rank of
+// a pair inside its expert group is the number of earlier pairs with the same expert
+// (a stable counting sort), so every index is uniquely defined and reproducible.
+#include "cep_common.h"
+
+namespace cep {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ int load_pair_id(const BatchDesc& b, int k, int p /*batch pair index*/) {
+  const int t = p / k;
+  int c = 0;
+#pragma unroll 1
+  while (c + 1 < b.n_chunks && t >= b.chunk[c + 1].token_base) ++c;
+  const long long off = (long long)(t - b.chunk[c].token_base) * k + (p - t * k);
+  return __ldg(b.chunk[c].ids + off);
+}
+
+// ---- 1. histogram: per segment of kSegPairs pairs, per local expert
+__global__ void __launch_bounds__(kThreads)
+hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global, int32_t* __restrict__ seg_hist,
+            int32_t* __restrict__ status) {
+  extern __shared__ int32_t sh[];
+  for (int e = threadIdx.x; e < E; e += kThreads) sh[e] = 0;
+  __syncthreads();
+  const int n_pairs = batch.n_tokens * k;
+  const int p0 = blockIdx.x * kSegPairs;
+  const int p1 = min(p0 + kSegPairs, n_pairs);
+  bool bad = false;
+  for (int p = p0 + threadIdx.x; p < p1; p += kThreads) {
+    const int e = load_pair_id(batch, k, p);
+    if (e < 0 || e >= E_global) bad = true;
+    else if (e < E) atomicAdd(&sh[e], 1);
+  }
+  if (bad) atomicOr(&status[kStBadRouting], 1);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += kThreads) seg_hist[(size_t)blockIdx.x * E + e] = sh[e];
+}
+
+// ---- 2. scan: counts, offsets, tile-aligned offsets, tile prefix, and per (segment, expert) row base
+__global__ void __launch_bounds__(1024)
+scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: row base*/,
+            int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ padded_offsets,
+            int32_t* __restrict__ tile_prefix) {
+  __shared__ int32_t s_cnt[1024];
+  __shared__ int32_t s_off[1025], s_pad[1025];
+  const int e = threadIdx.x;
+  int total = 0;
+  if (e < E) {
+    for (int s = 0; s < n_seg; ++s) {
+      const int c = seg_hist[(size_t)s * E + e];
+      seg_hist[(size_t)s * E + e] = total;      // exclusive prefix over segments
+      total += c;
+    }
+  }
+  s_cnt[e] = (e < E) ? total : 0;
+  __syncthreads();
+  if (threadIdx.x == 0) {                       // E <= 1024: a serial scan costs about a microsecond
+    int o = 0, po = 0;
+    for (int i = 0; i < E; ++i) {
+      s_off[i] = o; s_pad[i] = po;
+      o += s_cnt[i];
+      po += (s_cnt[i] + kRowAlign - 1) / kRowAlign * kRowAlign;
+    }
+    s_off[E] = o; s_pad[E] = po;
+  }
+  __syncthreads();
+  if (e < E) {
+    counts[e] = s_cnt[e];
+    offsets[e] = s_off[e];
+    padded_offsets[e] = s_pad[e];
+    tile_prefix[e] = s_pad[e] / kRowAlign;
+    const int base = s_pad[e];
+    for (int s = 0; s < n_seg; ++s) seg_hist[(size_t)s * E + e] += base;
+  }
+  if (e == 0) {
+    offsets[E] = s_off[E];
+    padded_offsets[E] = s_pad[E];
+    tile_prefix[E] = s_pad[E] / kRowAlign;
+  }
+}
+
+// ---- 3. stable rank: physical row of every pair, and the inverse map
+__global__ void __launch_bounds__(kThreads)
+rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t* __restrict__ seg_base,
+            int32_t* __restrict__ row_of_pair, int32_t* __restrict__ pair_of_row, int cap_rows,
+            int32_t* __restrict__ status) {
+  extern __shared__ int32_t sh[];              // [kWarps][E] running row cursor per warp and expert
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < kWarps * E; i += kThreads) sh[i] = 0;
+  __syncthreads();
+  const int n_pairs = batch.n_tokens * k;
+  constexpr int kPerWarp = kSegPairs / kWarps;
+  const int w0 = blockIdx.x * kSegPairs + warp * kPerWarp;
+  int32_t* mine = sh + warp * E;
+  // pass 1: this warp's count per expert
+  for (int it = 0; it < kPerWarp; it += 32) {
+    const int p = w0 + it + lane;
+    int e = -2;
+    if (p < n_pairs) { e = load_pair_id(batch, k, p); if (e < 0 || e >= E) e = -1; }
+    const unsigned m = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && lane == (__ffs(m) - 1)) mine[e] += __popc(m);
+    __syncwarp();
+  }
+  __syncthreads();
+  // exclusive prefix over the warps of this block, on top of the segment's row base
+  for (int e = threadIdx.x; e < E; e += kThreads) {
+    int run = seg_base[(size_t)blockIdx.x * E + e];
+    for (int w = 0; w < kWarps; ++w) { const int c = sh[w * E + e]; sh[w * E + e] = run; run += c; }
+  }
+  __syncthreads();
+  // pass 2: rows in pair order
+  for (int it = 0; it < kPerWarp; it += 32) {
+    const int p = w0 + it + lane;
+    int e = -2;
+    if (p < n_pairs) { e = load_pair_id(batch, k, p); if (e < 0 || e >= E) e = -1; }
+    const unsigned m = __match_any_sync(0xffffffffu, e);
+    int row = -1;
+    if (e >= 0) row = mine[e] + __popc(m & ((1u << lane) - 1u));
+    __syncwarp();
+    if (e >= 0 && lane == (__ffs(m) - 1)) mine[e] += __popc(m);
+    __syncwarp();
+    if (p < n_pairs) {
+      if (row >= cap_rows) { atomicOr(&status[kStBoundsViolation], 1); row = -1; }
+      row_of_pair[p] = row;
+      if (row >= 0) pair_of_row[row] = p;
+    }
+  }
+}
+
+// ---- 4. payload: one block per token reads its row once and writes it to each local expert's group;
+//         E extra blocks zero the padding rows of each group.
+template <int kVecPerThread>
+__global__ void __launch_bounds__(kThreads)
+scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int row_bytes, int n_scale,
+                    const int32_t* __restrict__ row_of_pair, const int32_t* __restrict__ counts,
+                    const int32_t* __restrict__ padded_offsets, int32_t* __restrict__ pair_of_row,
+                    uint8_t* __restrict__ xp, float* __restrict__ xp_scales, int cap_rows) {
+  const int n_vec = row_bytes >> 4;
+  if ((int)blockIdx.x >= batch.n_tokens) {       // padding rows of expert e
+    const int e = blockIdx.x - batch.n_tokens;
+    if (e >= E) return;
+    const int r0 = padded_offsets[e] + counts[e], r1 = padded_offsets[e + 1];
+    for (int r = r0; r < r1 && r < cap_rows; ++r) {
+      uint4* dst = reinterpret_cast<uint4*>(xp + (size_t)r * row_bytes);
+      for (int v = threadIdx.x; v < n_vec; v += kThreads) dst[v] = make_uint4(0, 0, 0, 0);
+      if (xp_scales) for (int v = threadIdx.x; v < n_scale; v += kThreads) xp_scales[(size_t)r * n_scale + v] = 0.f;
+      if (threadIdx.x == 0) pair_of_row[r] = -1;
+    }
+    return;
+  }
+  __shared__ int32_t s_rows[32];
+  const int t = blockIdx.x;
+  int c = 0;
+  while (c + 1 < batch.n_chunks && t >= batch.chunk[c + 1].token_base) ++c;
+  const int tl = t - batch.chunk[c].token_base;
+  if (threadIdx.x < k) s_rows[threadIdx.x] = row_of_pair[(size_t)t * k + threadIdx.x];
+  __syncthreads();
+  const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(batch.chunk[c].tokens) +
+                                                    (size_t)tl * row_bytes);
+  for (int v0 = threadIdx.x; v0 < n_vec; v0 += kThreads * kVecPerThread) {
+    uint4 val[kVecPerThread];
+#pragma unroll
+    for (int i = 0; i < kVecPerThread; ++i) {
+      const int v = v0 + i * kThreads;
+      if (v < n_vec) val[i] = __ldg(src + v);
+    }
+    for (int j = 0; j < k; ++j) {
+      const int row = s_rows[j];
+      if (row < 0) continue;
+      uint4* dst = reinterpret_cast<uint4*>(xp + (size_t)row * row_bytes);
+#pragma unroll
+      for (int i = 0; i < kVecPerThread; ++i) {
+        const int v = v0 + i * kThreads;
+        if (v < n_vec) dst[v] = val[i];
+      }
+    }
+  }
+  if (xp_scales) {
+    const float* ss = batch.chunk[c].scales + (size_t)tl * n_scale;
+    for (int v = threadIdx.x; v < n_scale; v += kThreads) {
+      const float sv = __ldg(ss + v);
+      for (int j = 0; j < k; ++j) {
+        const int row = s_rows[j];
+        if (row >= 0) xp_scales[(size_t)row * n_scale + v] = sv;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
+                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, int64_t* launches) {
+  const int k = cfg.top_k, E = cfg.n_experts_local;
+  if (n_seg < 1) n_seg = 1;
+  hist_kernel<<<n_seg, kThreads, E * sizeof(int32_t), s>>>(batch, k, E, cfg.n_experts_global, lp.block_base,
+                                                           lp.status);
+  scan_kernel<<<1, 1024, 0, s>>>(n_seg, E, lp.block_base, lp.counts, lp.offsets, lp.padded_offsets,
+                                 lp.tile_prefix);
+  rank_kernel<<<n_seg, kThreads, kWarps * E * sizeof(int32_t), s>>>(batch, k, E, lp.block_base, lp.row_of_pair,
+                                                                   lp.pair_of_row, cap_rows, lp.status);
+  const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128;
+  const int row_bytes = cfg.hidden * (fp8 ? 1 : 2);
+  const int n_scale = fp8 ? cfg.hidden / kQuantBlock : 0;
+  scatter_rows_kernel<4><<<batch.n_tokens + E, kThreads, 0, s>>>(
+      batch, k, E, row_bytes, n_scale, lp.row_of_pair, lp.counts, lp.padded_offsets, lp.pair_of_row,
+      static_cast<uint8_t*>(xp), fp8 ? xp_scales : nullptr, cap_rows);
+  *launches += 4;
+  return cudaGetLastError();
+}
+
+}  // namespace cep

@@ -1,0 +1,507 @@
+// Host runtime of the streamFFN library: plan object, workspace carving, the streamFFN
+// accumulator (threshold batching, final flush, round-robin streams; Section 3.2) and the
+// C ABI declared in include/cascade_ffn.h.  Host code only enqueues; it never waits for
+// the device except in ffn_debug_export / ffn_query / moe_plan_destroy.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cep_common.h"
+#include "gemm_tcgen05.h"
+
+using namespace cep;
+
+namespace {
+
+char g_error[256] = "";
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Slot {
+  LayoutPtrs lp;
+  uint8_t* xp; float* xp_scales;
+  uint8_t* act; float* act_scales;
+  uint8_t* y;
+  GemmTensorMap tm_a1, tm_a2;
+};
+
+struct Invocation {
+  int first_pos, n_chunks, slot, n_tokens;
+  int64_t pairs_bound;
+  cudaEvent_t start, done;
+};
+
+struct PendingChunk {
+  ChunkDesc d;
+  int64_t pairs;
+  int chunk_id;
+};
+
+// The launch rule, shared by the live path and cep_debug_schedule.
+bool should_launch(int mode, int64_t pending_pairs, int pending_chunks, int64_t theta) {
+  if (pending_chunks <= 0) return false;
+  if (pending_chunks >= kMaxChunksPerInv) return true;
+  if (mode == CEP_MODE_ASYNC) return true;
+  if (mode == CEP_MODE_STREAMFFN) return pending_pairs >= theta;
+  return false;                                   // CEP_MODE_SYNC: only at flush
+}
+
+struct Layout {                                   // byte offsets inside the workspace
+  size_t status;
+  size_t slot0, slot_bytes;
+  size_t counts, offsets, padded, tile_prefix, block_base, row_of_pair, pair_of_row, xp, xp_scales, act,
+      act_scales, y;                              // offsets inside a slot
+  size_t total;
+  int cap_rows, n_seg_max;
+};
+
+int validate(const cep_config* c, const char** why) {
+  *why = nullptr;
+  if (!c) { *why = "config is NULL"; return CEP_ERR_ARG; }
+  if (c->dtype != CEP_BF16 && c->dtype != CEP_FP8_E4M3_BLOCK128) { *why = "unknown dtype"; return CEP_ERR_ARG; }
+  if (c->hidden <= 0 || c->inter <= 0 || c->hidden % 128 || c->inter % 128) {
+    *why = "hidden and inter must be positive multiples of 128"; return CEP_ERR_ARG; }
+  if (c->n_experts_local <= 0 || c->n_experts_local > 1024 || c->n_experts_global < c->n_experts_local) {
+    *why = "need 0 < n_experts_local <= min(1024, n_experts_global)"; return CEP_ERR_ARG; }
+  if (c->top_k <= 0 || c->top_k > 32 || c->top_k > c->n_experts_global) { *why = "need 0 < top_k <= 32"; return CEP_ERR_ARG; }
+  if (c->max_tokens <= 0 || c->max_chunks <= 0) { *why = "max_tokens and max_chunks must be positive"; return CEP_ERR_ARG; }
+  if ((long long)c->max_tokens * c->top_k > (1ll << 30)) { *why = "max_tokens*top_k exceeds 2^30"; return CEP_ERR_ARG; }
+  if (c->mode < CEP_MODE_SYNC || c->mode > CEP_MODE_STREAMFFN) { *why = "unknown mode"; return CEP_ERR_ARG; }
+  if (c->n_streams < 1 || c->n_streams > 16) { *why = "n_streams must be in 1..16"; return CEP_ERR_ARG; }
+  if (c->threshold_pairs < 0) { *why = "threshold_pairs must be >= 0"; return CEP_ERR_ARG; }
+  if (c->gemm_impl != CEP_GEMM_TCGEN05 && c->gemm_impl != CEP_GEMM_SIMT) { *why = "unknown gemm_impl"; return CEP_ERR_ARG; }
+  return CEP_OK;
+}
+
+Layout make_layout(const cep_config& c) {
+  Layout L{};
+  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+  const size_t elt = fp8 ? 1 : 2;
+  const long long max_pairs = (long long)c.max_tokens * c.top_k;
+  const long long pad_groups = c.n_experts_local < max_pairs ? c.n_experts_local : max_pairs;
+  L.cap_rows = (int)align_up((size_t)(max_pairs + (kRowAlign - 1) * pad_groups), kRowAlign);
+  L.n_seg_max = (int)((max_pairs + kSegPairs - 1) / kSegPairs);
+  if (L.n_seg_max < 1) L.n_seg_max = 1;
+  const size_t E = c.n_experts_local, A = 256;
+  size_t o = 0;
+  L.counts = o; o = align_up(o + E * 4, A);
+  L.offsets = o; o = align_up(o + (E + 1) * 4, A);
+  L.padded = o; o = align_up(o + (E + 1) * 4, A);
+  L.tile_prefix = o; o = align_up(o + (E + 1) * 4, A);
+  L.block_base = o; o = align_up(o + (size_t)L.n_seg_max * E * 4, A);
+  L.row_of_pair = o; o = align_up(o + (size_t)max_pairs * 4, A);
+  L.pair_of_row = o; o = align_up(o + (size_t)L.cap_rows * 4, A);
+  L.xp = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.hidden * elt, A);
+  L.xp_scales = o; o = align_up(o + (fp8 ? (size_t)L.cap_rows * (c.hidden / kQuantBlock) * 4 : 0), A);
+  L.act = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.inter * elt, A);
+  L.act_scales = o; o = align_up(o + (fp8 ? (size_t)L.cap_rows * (c.inter / kQuantBlock) * 4 : 0), A);
+  L.y = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.hidden * 2, 1024);
+  L.slot_bytes = o;
+  L.status = 0;
+  L.slot0 = 1024;
+  L.total = L.slot0 + L.slot_bytes * c.n_streams;
+  return L;
+}
+
+struct PackedLayout { size_t w13, w2, s13, s2, total; };
+PackedLayout make_packed_layout(const cep_config& c) {
+  PackedLayout P{};
+  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+  const size_t elt = fp8 ? 1 : 2, E = c.n_experts_local, H = c.hidden, I = c.inter;
+  size_t o = 0;
+  P.w13 = o; o = align_up(o + E * 2 * I * H * elt, 1024);
+  P.w2 = o; o = align_up(o + E * H * I * elt, 1024);
+  P.s13 = o; o = align_up(o + (fp8 ? E * (2 * I / kQuantBlock) * (H / kQuantBlock) * 4 : 0), 1024);
+  P.s2 = o; o = align_up(o + (fp8 ? E * (H / kQuantBlock) * (I / kQuantBlock) * 4 : 0), 1024);
+  P.total = o;
+  return P;
+}
+
+}  // namespace
+
+struct cep_plan {
+  cep_config cfg;
+  Layout L;
+  uint8_t* ws;
+  int n_sms;
+  std::vector<cudaStream_t> streams;
+  std::vector<Slot> slots;
+  std::vector<cudaEvent_t> ready_evt;           // per chunk position
+  std::vector<Invocation> inv;
+  std::vector<cudaEvent_t> inv_start, inv_done; // pools, one per possible invocation
+  cudaEvent_t begin_evt, readback_evt, weights_evt;
+  bool have_weights, layer_open, flushed, readback_pending, ever_closed;
+  uint8_t* w13p; uint8_t* w2p;
+  GemmTensorMap tm_b1, tm_b2;
+  // current layer call
+  void* out; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
+  std::vector<char> chunk_seen;
+  std::vector<PendingChunk> pending;
+  int64_t pending_pairs;
+  int32_t* host_status;                         // pinned
+  int64_t launches;
+  char err[256];
+};
+
+namespace {
+
+int fail(cep_plan* p, int code, const char* fmt, ...) {
+  char* dst = p ? p->err : g_error;
+  va_list ap; va_start(ap, fmt); vsnprintf(dst, 256, fmt, ap); va_end(ap);
+  return code;
+}
+#define CUDA_TRY(p, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) \
+  return fail((p), CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); } while (0)
+
+int launch_invocation(cep_plan* p) {
+  if (p->pending.empty()) return CEP_OK;
+  const cep_config& c = p->cfg;
+  const int idx = (int)p->inv.size();
+  if (idx >= (int)p->inv_start.size()) return fail(p, CEP_ERR_CAPACITY, "more invocations than max_chunks");
+  const int slot_i = idx % c.n_streams;
+  Slot& sl = p->slots[slot_i];
+  cudaStream_t st = p->streams[slot_i];
+  BatchDesc batch{};
+  int tok = 0;
+  const int first_pos = p->n_submitted - (int)p->pending.size();
+  for (size_t i = 0; i < p->pending.size(); ++i) {
+    batch.chunk[i] = p->pending[i].d;
+    batch.chunk[i].token_base = tok;
+    tok += p->pending[i].d.n_tokens;
+  }
+  batch.n_chunks = (int)p->pending.size();
+  batch.n_tokens = tok;
+  CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
+  CUDA_TRY(p, cudaStreamWaitEvent(st, p->weights_evt, 0));
+  for (size_t i = 0; i < p->pending.size(); ++i) CUDA_TRY(p, cudaStreamWaitEvent(st, p->ready_evt[first_pos + (int)i], 0));
+  Invocation iv{first_pos, batch.n_chunks, slot_i, tok, p->pending_pairs, p->inv_start[idx], p->inv_done[idx]};
+  CUDA_TRY(p, cudaEventRecord(iv.start, st));
+  if (tok > 0) {
+    const long long n_pairs = (long long)tok * c.top_k;
+    const int n_seg = (int)((n_pairs + kSegPairs - 1) / kSegPairs);
+    CUDA_TRY(p, launch_layout(batch, c, sl.lp, sl.xp, sl.xp_scales, p->L.cap_rows, n_seg, st, &p->launches));
+    const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+    const long long groups = c.n_experts_local < n_pairs ? c.n_experts_local : n_pairs;
+    const long long m_tiles_bound = (n_pairs + (kRowAlign - 1) * groups + kRowAlign - 1) / kRowAlign;
+    GemmProblem g1{c.hidden, 2 * c.inter, c.n_experts_local, 1, c.inter, p->L.cap_rows, fp8};
+    GemmProblem g2{c.inter, c.hidden, c.n_experts_local, 0, c.hidden, p->L.cap_rows, fp8};
+    if (c.gemm_impl == CEP_GEMM_SIMT) {
+      CUDA_TRY(p, launch_gemm_simt(g1, sl.xp, p->w13p, sl.act, sl.lp, st, &p->launches));
+      CUDA_TRY(p, launch_gemm_simt(g2, sl.act, p->w2p, sl.y, sl.lp, st, &p->launches));
+    } else {
+      const int bn = gemm_tile_cols();
+      const long long t1 = m_tiles_bound * ((g1.N + bn - 1) / bn), t2 = m_tiles_bound * ((g2.N + bn - 1) / bn);
+      CUDA_TRY(p, launch_gemm_tcgen05(g1, sl.tm_a1, p->tm_b1, sl.act, sl.lp, (int)(t1 > (1 << 30) ? (1 << 30) : t1),
+                                      p->n_sms, st, &p->launches));
+      CUDA_TRY(p, launch_gemm_tcgen05(g2, sl.tm_a2, p->tm_b2, sl.y, sl.lp, (int)(t2 > (1 << 30) ? (1 << 30) : t2),
+                                      p->n_sms, st, &p->launches));
+    }
+    CUDA_TRY(p, launch_combine(batch, c, sl.lp, sl.y, p->out, st, &p->launches));
+  }
+  CUDA_TRY(p, cudaEventRecord(iv.done, st));
+  p->inv.push_back(iv);
+  p->pending.clear();
+  p->pending_pairs = 0;
+  return CEP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cep_last_error(const cep_plan* plan) { return plan ? plan->err : g_error; }
+
+int moe_plan_workspace_bytes(const cep_config* cfg, size_t* bytes) {
+  const char* why;
+  int rc = validate(cfg, &why);
+  if (rc) return fail(nullptr, rc, "%s", why);
+  if (!bytes) return fail(nullptr, CEP_ERR_ARG, "bytes is NULL");
+  *bytes = make_layout(*cfg).total;
+  return CEP_OK;
+}
+
+int moe_packed_weight_bytes(const cep_config* cfg, size_t* bytes) {
+  const char* why;
+  int rc = validate(cfg, &why);
+  if (rc) return fail(nullptr, rc, "%s", why);
+  if (!bytes) return fail(nullptr, CEP_ERR_ARG, "bytes is NULL");
+  *bytes = make_packed_layout(*cfg).total;
+  return CEP_OK;
+}
+
+int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep_plan** out) {
+  const char* why;
+  int rc = validate(cfg, &why);
+  if (rc) return fail(nullptr, rc, "%s", why);
+  if (!out) return fail(nullptr, CEP_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (!workspace) return fail(nullptr, CEP_ERR_ARG, "workspace is NULL");
+  if (cfg->dtype == CEP_FP8_E4M3_BLOCK128)
+    return fail(nullptr, CEP_ERR_UNSUPPORTED, "the block-scaled fp8 path is not built yet");
+  Layout L = make_layout(*cfg);
+  if (workspace_bytes < L.total) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+  if (reinterpret_cast<uintptr_t>(workspace) % 256) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+  cep_plan* p = new (std::nothrow) cep_plan();
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "out of host memory");
+  p->cfg = *cfg; p->L = L; p->ws = static_cast<uint8_t*>(workspace);
+  p->err[0] = 0; p->launches = 0;
+  p->have_weights = p->layer_open = p->flushed = p->readback_pending = p->ever_closed = false;
+  p->host_status = nullptr; p->begin_evt = p->readback_evt = p->weights_evt = nullptr;
+  p->out = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
+  int dev = 0;
+#define PLAN_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
+    fail(nullptr, CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); moe_plan_destroy(p); return CEP_ERR_CUDA; } } while (0)
+  PLAN_TRY(cudaGetDevice(&dev));
+  PLAN_TRY(cudaDeviceGetAttribute(&p->n_sms, cudaDevAttrMultiProcessorCount, dev));
+  PLAN_TRY(cudaHostAlloc(reinterpret_cast<void**>(&p->host_status), kStWords * sizeof(int32_t), cudaHostAllocDefault));
+  memset(p->host_status, 0, kStWords * sizeof(int32_t));
+  PLAN_TRY(cudaEventCreateWithFlags(&p->begin_evt, cudaEventDisableTiming));
+  PLAN_TRY(cudaEventCreateWithFlags(&p->readback_evt, cudaEventDisableTiming));
+  PLAN_TRY(cudaEventCreateWithFlags(&p->weights_evt, cudaEventDisableTiming));
+  for (int s = 0; s < cfg->n_streams; ++s) {
+    cudaStream_t st;
+    PLAN_TRY(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+    p->streams.push_back(st);
+  }
+  for (int i = 0; i < cfg->max_chunks; ++i) {
+    cudaEvent_t e;
+    PLAN_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming)); p->ready_evt.push_back(e);
+    PLAN_TRY(cudaEventCreate(&e)); p->inv_start.push_back(e);
+    PLAN_TRY(cudaEventCreate(&e)); p->inv_done.push_back(e);
+  }
+  const bool fp8 = cfg->dtype == CEP_FP8_E4M3_BLOCK128;
+  const int elt = fp8 ? 1 : 2;
+  for (int s = 0; s < cfg->n_streams; ++s) {
+    uint8_t* b = p->ws + L.slot0 + L.slot_bytes * s;
+    Slot sl{};
+    sl.lp.counts = reinterpret_cast<int32_t*>(b + L.counts);
+    sl.lp.offsets = reinterpret_cast<int32_t*>(b + L.offsets);
+    sl.lp.padded_offsets = reinterpret_cast<int32_t*>(b + L.padded);
+    sl.lp.tile_prefix = reinterpret_cast<int32_t*>(b + L.tile_prefix);
+    sl.lp.block_base = reinterpret_cast<int32_t*>(b + L.block_base);
+    sl.lp.row_of_pair = reinterpret_cast<int32_t*>(b + L.row_of_pair);
+    sl.lp.pair_of_row = reinterpret_cast<int32_t*>(b + L.pair_of_row);
+    sl.lp.status = reinterpret_cast<int32_t*>(p->ws + L.status);
+    sl.xp = b + L.xp; sl.xp_scales = reinterpret_cast<float*>(b + L.xp_scales);
+    sl.act = b + L.act; sl.act_scales = reinterpret_cast<float*>(b + L.act_scales);
+    sl.y = b + L.y;
+    if (cfg->gemm_impl == CEP_GEMM_TCGEN05) {
+      int r1 = make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
+      int r2 = make_operand_map(&sl.tm_a2, sl.act, elt, cfg->inter, L.cap_rows, 0, gemm_tile_rows());
+      if (r1 || r2) {
+        fail(nullptr, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the activation operands failed (%d, %d)", r1, r2);
+        moe_plan_destroy(p);
+        return CEP_ERR_CUDA;
+      }
+    }
+    p->slots.push_back(sl);
+  }
+  // status word starts clean
+  PLAN_TRY(cudaMemsetAsync(p->ws + L.status, 0, kStWords * sizeof(int32_t), p->streams[0]));
+  PLAN_TRY(cudaEventRecord(p->begin_evt, p->streams[0]));
+  PLAN_TRY(cudaEventRecord(p->weights_evt, p->streams[0]));
+#undef PLAN_TRY
+  *out = p;
+  return CEP_OK;
+}
+
+int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const void* w_down, const float* s_gate,
+                     const float* s_up, const float* s_down, void* packed, size_t packed_bytes, void* stream) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!w_gate || !w_up || !w_down || !packed) return fail(p, CEP_ERR_ARG, "a weight pointer is NULL");
+  if (p->layer_open) return fail(p, CEP_ERR_STATE, "weights cannot change while a layer call is open");
+  const cep_config& c = p->cfg;
+  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+  if (fp8 && (!s_gate || !s_up || !s_down)) return fail(p, CEP_ERR_ARG, "fp8 weights need their scale tensors");
+  PackedLayout P = make_packed_layout(c);
+  if (packed_bytes < P.total) return fail(p, CEP_ERR_WORKSPACE, "packed buffer has %zu bytes, %zu needed", packed_bytes, P.total);
+  if (reinterpret_cast<uintptr_t>(packed) % 256) return fail(p, CEP_ERR_WORKSPACE, "packed buffer must be 256-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  p->w13p = static_cast<uint8_t*>(packed) + P.w13;
+  p->w2p = static_cast<uint8_t*>(packed) + P.w2;
+  CUDA_TRY(p, launch_prepack(c, w_gate, w_up, w_down, p->w13p, p->w2p, st, &p->launches));
+  CUDA_TRY(p, cudaEventRecord(p->weights_evt, st));
+  if (c.gemm_impl == CEP_GEMM_TCGEN05) {
+    const int elt = fp8 ? 1 : 2;
+    int r1 = make_operand_map(&p->tm_b1, p->w13p, elt, c.hidden, 2 * c.inter, c.n_experts_local, gemm_tile_cols());
+    int r2 = make_operand_map(&p->tm_b2, p->w2p, elt, c.inter, c.hidden, c.n_experts_local, gemm_tile_cols());
+    if (r1 || r2) return fail(p, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the weight operands failed (%d, %d)", r1, r2);
+  }
+  p->have_weights = true;
+  return CEP_OK;
+}
+
+int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_expected) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_begin while a layer call is open (call combine first)");
+  if (!p->have_weights) return fail(p, CEP_ERR_STATE, "ffn_begin before moe_load_weights");
+  if (!out || n_tokens_total < 0 || n_chunks_expected < 0) return fail(p, CEP_ERR_ARG, "bad ffn_begin arguments");
+  if (n_tokens_total > p->cfg.max_tokens) return fail(p, CEP_ERR_CAPACITY, "%d tokens, plan made for %d", n_tokens_total, p->cfg.max_tokens);
+  if (n_chunks_expected > p->cfg.max_chunks) return fail(p, CEP_ERR_CAPACITY, "%d chunks, plan made for %d", n_chunks_expected, p->cfg.max_chunks);
+  cudaStream_t s0 = p->streams[0];
+  // the previous layer's status read-back must finish before the status word is cleared
+  if (p->readback_pending) CUDA_TRY(p, cudaStreamWaitEvent(s0, p->readback_evt, 0));
+  CUDA_TRY(p, cudaMemsetAsync(p->ws + p->L.status, 0, kStWords * sizeof(int32_t), s0));
+  CUDA_TRY(p, cudaEventRecord(p->begin_evt, s0));
+  p->out = out; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
+  p->n_submitted = 0; p->tokens_submitted = 0;
+  p->chunk_seen.assign(n_chunks_expected, 0);
+  p->pending.clear(); p->pending_pairs = 0; p->inv.clear();
+  p->layer_open = true; p->flushed = false;
+  return CEP_OK;
+}
+
+int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_t n_tokens, const void* tokens,
+                     const float* token_scales, const int32_t* topk_ids, const float* topk_weights,
+                     int64_t n_local_pairs, void* stream) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_submit_chunk before ffn_begin");
+  if (p->flushed) return fail(p, CEP_ERR_STATE, "ffn_submit_chunk after ffn_flush");
+  if (chunk_id < 0 || chunk_id >= p->n_chunks_expected) return fail(p, CEP_ERR_ARG, "chunk_id %d outside 0..%d", chunk_id, p->n_chunks_expected - 1);
+  if (p->chunk_seen[chunk_id]) return fail(p, CEP_ERR_STATE, "chunk %d submitted twice", chunk_id);
+  if (n_tokens < 0 || token_offset < 0) return fail(p, CEP_ERR_ARG, "negative n_tokens or token_offset");
+  if ((long long)token_offset + n_tokens > p->n_tokens_total) return fail(p, CEP_ERR_CAPACITY, "chunk %d covers tokens beyond n_tokens_total", chunk_id);
+  if (n_tokens > 0 && (!tokens || !topk_ids || !topk_weights)) return fail(p, CEP_ERR_ARG, "a chunk pointer is NULL");
+  const bool fp8 = p->cfg.dtype == CEP_FP8_E4M3_BLOCK128;
+  if (fp8 && n_tokens > 0 && !token_scales) return fail(p, CEP_ERR_ARG, "fp8 chunk without token_scales");
+  const int64_t bound = (int64_t)n_tokens * p->cfg.top_k;
+  if (n_local_pairs > bound) return fail(p, CEP_ERR_ARG, "n_local_pairs exceeds n_tokens*top_k");
+  const int64_t pairs = n_local_pairs < 0 ? bound : n_local_pairs;
+  CUDA_TRY(p, cudaEventRecord(p->ready_evt[p->n_submitted], static_cast<cudaStream_t>(stream)));
+  PendingChunk pc{};
+  pc.d.tokens = tokens; pc.d.scales = token_scales; pc.d.ids = topk_ids; pc.d.weights = topk_weights;
+  pc.d.n_tokens = n_tokens; pc.d.token_offset = token_offset;
+  pc.pairs = pairs; pc.chunk_id = chunk_id;
+  p->pending.push_back(pc);
+  p->pending_pairs += pairs;
+  p->chunk_seen[chunk_id] = 1;
+  p->n_submitted += 1;
+  p->tokens_submitted += n_tokens;
+  if (should_launch(p->cfg.mode, p->pending_pairs, (int)p->pending.size(), p->cfg.threshold_pairs))
+    return launch_invocation(p);
+  return CEP_OK;
+}
+
+int ffn_flush(cep_plan* p) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_flush before ffn_begin");
+  p->flushed = true;
+  int rc = launch_invocation(p);
+  if (rc) return rc;
+  if (p->n_submitted < p->n_chunks_expected)
+    return fail(p, CEP_ERR_INCOMPLETE, "flush after %d of %d chunks", p->n_submitted, p->n_chunks_expected);
+  return CEP_OK;
+}
+
+int combine(cep_plan* p, void* stream) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->layer_open) return fail(p, CEP_ERR_STATE, "combine before ffn_begin");
+  int rc = CEP_OK;
+  if (!p->flushed) { rc = ffn_flush(p); if (rc && rc != CEP_ERR_INCOMPLETE) return rc; }
+  else if (p->n_submitted < p->n_chunks_expected)
+    rc = fail(p, CEP_ERR_INCOMPLETE, "combine after %d of %d chunks", p->n_submitted, p->n_chunks_expected);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
+  for (const Invocation& iv : p->inv) CUDA_TRY(p, cudaStreamWaitEvent(st, iv.done, 0));
+  CUDA_TRY(p, cudaMemcpyAsync(p->host_status, p->ws + p->L.status, kStWords * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(p, cudaEventRecord(p->readback_evt, st));
+  p->readback_pending = true; p->ever_closed = true;
+  p->layer_open = false;
+  return rc;
+}
+
+int ffn_status(cep_plan* p) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->ever_closed || p->layer_open) return fail(p, CEP_ERR_STATE, "no closed layer call to report on");
+  cudaError_t q = cudaEventQuery(p->readback_evt);
+  if (q == cudaErrorNotReady) return fail(p, CEP_ERR_STATE, "the stream given to combine has not completed yet");
+  if (q != cudaSuccess) return fail(p, CEP_ERR_CUDA, "cudaEventQuery failed: %s", cudaGetErrorString(q));
+  if (p->host_status[kStTimeout]) return fail(p, CEP_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired");
+  if (p->host_status[kStBoundsViolation]) return fail(p, CEP_ERR_CAPACITY, "a row index left the scratch slot (more local pairs than planned)");
+  if (p->host_status[kStBadRouting]) return fail(p, CEP_ERR_BAD_ROUTING, "an expert id was outside [0, n_experts_global)");
+  return CEP_OK;
+}
+
+int ffn_num_invocations(const cep_plan* p) { return p ? (int)p->inv.size() : CEP_ERR_ARG; }
+
+int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {
+  if (!p || !info) return fail(p, CEP_ERR_ARG, "NULL argument");
+  if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
+  const Invocation& iv = p->inv[inv];
+  info->n_chunks = iv.n_chunks; info->first_chunk_pos = iv.first_pos; info->stream_index = iv.slot;
+  info->n_tokens = iv.n_tokens; info->pairs_bound = iv.pairs_bound; info->elapsed_ms = -1.f;
+  if (cudaEventQuery(iv.done) == cudaSuccess) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, iv.start, iv.done) == cudaSuccess) info->elapsed_ms = ms;
+  }
+  return CEP_OK;
+}
+
+int ffn_debug_export(cep_plan* p, int32_t inv, int32_t* counts, int32_t* offsets, int32_t* padded_offsets,
+                     int32_t* row_of_pair, int32_t* pair_of_row) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
+  const Invocation& iv = p->inv[inv];
+  if ((int)p->inv.size() - inv > p->cfg.n_streams) return fail(p, CEP_ERR_STATE, "scratch slot of invocation %d was reused", inv);
+  CUDA_TRY(p, cudaEventSynchronize(iv.done));
+  const Slot& sl = p->slots[iv.slot];
+  const int E = p->cfg.n_experts_local;
+  std::vector<int32_t> po(E + 1, 0);
+  if (iv.n_tokens > 0) CUDA_TRY(p, cudaMemcpy(po.data(), sl.lp.padded_offsets, (E + 1) * 4, cudaMemcpyDeviceToHost));
+  if (iv.n_tokens == 0) {
+    if (counts) memset(counts, 0, E * 4);
+    if (offsets) memset(offsets, 0, (E + 1) * 4);
+    if (padded_offsets) memset(padded_offsets, 0, (E + 1) * 4);
+    return CEP_OK;
+  }
+  if (counts) CUDA_TRY(p, cudaMemcpy(counts, sl.lp.counts, E * 4, cudaMemcpyDeviceToHost));
+  if (offsets) CUDA_TRY(p, cudaMemcpy(offsets, sl.lp.offsets, (E + 1) * 4, cudaMemcpyDeviceToHost));
+  if (padded_offsets) memcpy(padded_offsets, po.data(), (E + 1) * 4);
+  if (row_of_pair) CUDA_TRY(p, cudaMemcpy(row_of_pair, sl.lp.row_of_pair, (size_t)iv.n_tokens * p->cfg.top_k * 4, cudaMemcpyDeviceToHost));
+  if (pair_of_row && po[E] > 0) CUDA_TRY(p, cudaMemcpy(pair_of_row, sl.lp.pair_of_row, (size_t)po[E] * 4, cudaMemcpyDeviceToHost));
+  return CEP_OK;
+}
+
+int64_t cep_kernel_launches(const cep_plan* p) { return p ? p->launches : 0; }
+
+int moe_plan_destroy(cep_plan* p) {
+  if (!p) return CEP_OK;
+  for (cudaStream_t s : p->streams) cudaStreamSynchronize(s);
+  for (cudaEvent_t e : p->ready_evt) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->inv_start) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->inv_done) cudaEventDestroy(e);
+  if (p->begin_evt) cudaEventDestroy(p->begin_evt);
+  if (p->readback_evt) { cudaEventSynchronize(p->readback_evt); cudaEventDestroy(p->readback_evt); }
+  if (p->weights_evt) cudaEventDestroy(p->weights_evt);
+  for (cudaStream_t s : p->streams) cudaStreamDestroy(s);
+  if (p->host_status) cudaFreeHost(p->host_status);
+  delete p;
+  return CEP_OK;
+}
+
+int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n, int32_t tile,
+                          int32_t* expert, int32_t* m_block, int32_t* n_block) {
+  if (!tile_prefix || n_experts <= 0 || !expert || !m_block || !n_block) return CEP_ERR_ARG;
+  TileCoord tc;
+  if (!decode_tile(tile_prefix, n_experts, n_blocks_n, tile, &tc)) return CEP_ERR_ARG;
+  *expert = tc.expert; *m_block = tc.m_block; *n_block = tc.n_block;
+  return CEP_OK;
+}
+
+int cep_debug_schedule(const int64_t* pairs, int32_t n_chunks, int32_t mode, int64_t theta,
+                       int32_t* invocation_of_chunk) {
+  if (n_chunks < 0 || (n_chunks > 0 && (!pairs || !invocation_of_chunk))) return CEP_ERR_ARG;
+  int inv = 0, pending = 0;
+  int64_t acc = 0;
+  for (int c = 0; c < n_chunks; ++c) {
+    invocation_of_chunk[c] = inv;
+    ++pending; acc += pairs[c];
+    if (should_launch(mode, acc, pending, theta)) { ++inv; pending = 0; acc = 0; }
+  }
+  if (pending) ++inv;                             // final flush
+  return inv;
+}
+
+}  // extern "C"
