@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the streamFFN routed-expert path on B200.
+
+One "step" = one pass of the whole hot path (layout transform, both expert GEMMs with the
+fused activation, weighted combine) over one batch of synthetic routed tokens, all chunks
+present, through the C ABI.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config ep_shard|mid|...]
+  python bench.py --impl reference ...     # times the CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MoE-layer prefill tokens/s (streamFFN routed-expert path: permute + grouped SwiGLU expert FFN + combine)"
+UNIT = "tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_numbers(cfg, n_pairs):
+    """Algorithmic work of one step ('Algorithmic work per unit')."""
+    H, I, T, E = cfg.H, cfg.I, cfg.T, cfg.E_local
+    s = 2
+    return {
+        "pairs": n_pairs,
+        "flops": 6.0 * H * I * n_pairs,
+        "gemm1_flops": 4.0 * H * I * n_pairs,
+        "gemm2_flops": 2.0 * H * I * n_pairs,
+        "layout_bytes": (T + n_pairs) * H * s + T * cfg.k * 4.0,
+        "combine_bytes": (n_pairs + T) * H * 2.0 + n_pairs * 4.0,
+        "gemm1_bytes": n_pairs * H * s + 2.0 * H * I * s * E + n_pairs * I * s,
+        "gemm2_bytes": n_pairs * I * s + 1.0 * H * I * s * E + n_pairs * H * 2,
+    }
+
+
+def host_copy(inp):
+    """The same inputs with every tensor on the host (for the CPU oracle)."""
+    import dataclasses
+    import torch
+    kw = {}
+    for f in dataclasses.fields(inp):
+        v = getattr(inp, f.name)
+        kw[f.name] = v.cpu() if isinstance(v, torch.Tensor) else v
+    return type(inp)(**kw)
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    import numpy as np
+    import oracle
+    from paper_2609_33252_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import torch
+    cfg = wl.CONFIGS[args.config]
+    n_sample = args.oracle_tokens
+    inp = wl.make_inputs(cfg, device="cuda" if torch.cuda.is_available() else "cpu", keep_logits=False)
+    inp = host_copy(inp)
+    cores = oracle.num_threads()
+    sel = np.linspace(0, cfg.T - 1, n_sample).astype(np.int64)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oracle.from_inputs(inp, sel=sel)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    dt = sum(times) / len(times)
+    val = n_sample / dt
+    sample = "%d evenly spaced tokens of the %s workload, all their local routed pairs, fp64" % (n_sample, cfg.name)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E_local": cfg.E_local,
+                       "E_global": cfg.E_global, "top_k": cfg.k, "sample_tokens": n_sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="ep_shard")
+    ap.add_argument("--streams", type=int, default=2)
+    ap.add_argument("--oracle-tokens", type=int, default=48)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3 if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        if args.steps > 3:
+            args.steps = 3
+        args.warmup = min(args.warmup, 1)
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import paper_2609_33252_b200 as cep
+    from paper_2609_33252_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg = wl.CONFIGS[args.config]
+    peaks = load_peaks()
+    inp = wl.make_inputs(cfg, device="cuda", keep_logits=False)
+    n_pairs = inp.n_local_pairs()
+    work = workload_numbers(cfg, n_pairs)
+    ch_pairs = [int((inp.topk_ids[o:o + n] < cfg.E_local).sum().item()) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
+
+    layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks,
+                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, profile_kernels=1)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+    torch.cuda.synchronize()
+    out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
+    chunks = [(o, inp.x[o:o + n], None if inp.x_scale is None else inp.x_scale[o:o + n], inp.topk_ids[o:o + n],
+               inp.topk_w[o:o + n]) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
+
+    def step():
+        layer.run(out, chunks, n_local_pairs=ch_pairs)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = cep.cep_kernel_launches(layer.plan)
+    kern = {"layout_ms": [], "gemm1_ms": [], "gemm2_ms": [], "combine_ms": []}
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+        # per-kernel device times of this step's invocations are read after the timed region;
+        # the plan keeps only the last layer call, so collect lazily below
+    ev1.record()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    launches = cep.cep_kernel_launches(layer.plan) - launches0
+    assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
+    # per-kernel times: a few more steps, each followed by a sync and a query (outside the timed region)
+    for _ in range(min(args.steps, 5)):
+        step()
+        torch.cuda.synchronize()
+        for i in range(cep.ffn_num_invocations(layer.plan)):
+            info = cep.ffn_query(layer.plan, i)
+            for k_ in kern:
+                kern[k_].append(getattr(info, k_))
+    clocks = sampler.stop() if rank == 0 else None
+    ms = total_ms / args.steps
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * cfg.T / (ms * 1e-3)
+
+    # ---- end to end: pinned host buffers -> device -> path -> host, every step
+    e2e = None
+    if not args.no_e2e:
+        hx = inp.x.cpu().pin_memory(); hid = inp.topk_ids.cpu().pin_memory(); hw = inp.topk_w.cpu().pin_memory()
+        hout = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory()
+        dx, did, dw = torch.empty_like(inp.x), torch.empty_like(inp.topk_ids), torch.empty_like(inp.topk_w)
+        rstreams = [torch.cuda.Stream() for _ in chunks]
+        main = torch.cuda.current_stream()
+
+        def e2e_step():
+            cep.ffn_begin(layer.plan, out, cfg.T, len(chunks))
+            for c, (o, n) in enumerate(zip(inp.chunk_offsets, cfg.chunks)):
+                st = rstreams[c]
+                st.wait_stream(main)
+                with torch.cuda.stream(st):
+                    dx[o:o + n].copy_(hx[o:o + n], non_blocking=True)
+                    did[o:o + n].copy_(hid[o:o + n], non_blocking=True)
+                    dw[o:o + n].copy_(hw[o:o + n], non_blocking=True)
+                cep.ffn_submit_chunk(layer.plan, c, o, n, dx[o:o + n], None, did[o:o + n], dw[o:o + n], ch_pairs[c], st)
+            cep.ffn_flush(layer.plan)
+            cep.combine(layer.plan, main)
+            hout.copy_(out, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        ev0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        ev1.record()
+        barrier()
+        e2e_ms = ev0.elapsed_time(ev1) / args.steps
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = hx.numel() * 2 + hid.numel() * 4 + hw.numel() * 4
+        e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": hout.numel() * 2}
+
+    if rank != 0:
+        layer.close()
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    med = {k_: (statistics.median(v) if v else None) for k_, v in kern.items()}
+    g1_ms, g2_ms = med["gemm1_ms"], med["gemm2_ms"]
+    ffn_tflops = work["flops"] / ((g1_ms + g2_ms) * 1e-3) / 1e12
+    g1_tflops = work["gemm1_flops"] / (g1_ms * 1e-3) / 1e12
+    g2_tflops = work["gemm2_flops"] / (g2_ms * 1e-3) / 1e12
+    sustained = ms > 5.0          # a step of several ms runs under the power cap
+    peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    roofline = {"bound": "tensor", "kernel": "grouped_gemm_bf16_kernel<swiglu> (GEMM1: gate/up + SiLU*up)",
+                "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
+                "peak_kind": ("sustained" if sustained else "burst") + " bf16 cuBLAS, of " + peaks["source"],
+                "frac_of_nominal_2250": g1_tflops / NOMINAL_BF16_TFLOPS,
+                "duration_ms": g1_ms, "traffic": None}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            tr = json.load(open(prof)).get(cfg.name, {})
+            roofline["traffic"] = tr.get("gemm1_dram_bytes_per_launch")
+        except Exception:
+            pass
+    kernels = {
+        "layout": {"ms": med["layout_ms"], "GB/s": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9,
+                   "frac_of_hbm": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "gemm1": {"ms": g1_ms, "TFLOP/s": g1_tflops},
+        "gemm2": {"ms": g2_ms, "TFLOP/s": g2_tflops, "frac": g2_tflops / peak_tf},
+        "combine": {"ms": med["combine_ms"], "GB/s": work["combine_bytes"] / (med["combine_ms"] * 1e-3) / 1e9,
+                    "frac_of_hbm": work["combine_bytes"] / (med["combine_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+    }
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "fp8_e4m3", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E_local": cfg.E_local,
+                       "E_global": cfg.E_global, "top_k": cfg.k, "local_pairs": n_pairs, "chunks": list(cfg.chunks),
+                       "mode": "sync (one invocation, all chunks present)", "parallelism": "replicas only",
+                       "l2": "inputs larger than L2 (weights %.2f GB re-read every step)" %
+                             (3.0 * cfg.H * cfg.I * 2 * cfg.E_local / 1e9)},
+            "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal_2250": ffn_tflops / NOMINAL_BF16_TFLOPS,
+                           "frac_of_measured": ffn_tflops / peak_tf, "flops_per_step": work["flops"]},
+            "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(launches)}
+    if not args.no_cpu_baseline:
+        import oracle
+        n_s = args.oracle_tokens
+        hin = host_copy(inp)
+        sel = np.linspace(0, cfg.T - 1, n_s).astype(np.int64)
+        t0 = time.perf_counter()
+        ref = oracle.from_inputs(hin, sel=sel)
+        dt = time.perf_counter() - t0
+        got = out[torch.as_tensor(sel, device="cuda")].double().cpu().numpy()
+        rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+        line["cpu_baseline"] = {"value": n_s / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": "%d evenly spaced tokens of the %s workload, all their local routed "
+                                          "pairs, fp64, %.1f s" % (n_s, cfg.name, dt),
+                                "rel_fro_error_of_gpu_on_sample": rel}
+    print(json.dumps(line))
+    layer.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -103,6 +103,9 @@ typedef struct {
   int32_t gemm_impl;           /* cep_gemm_impl                                                 */
   int32_t debug_checks;        /* nonzero: kernels bounds-check every index and record, never
                                   trap, on violation                                            */
+  int32_t profile_kernels;     /* nonzero: record CUDA events between the kernels of every
+                                  invocation so ffn_query can report per-kernel device times    */
+  int32_t reserved_;           /* set to 0                                                      */
 } cep_config;
 
 /* Per-invocation record for tracing (ffn_query). */
@@ -113,6 +116,10 @@ typedef struct {
   int32_t n_tokens;            /* tokens in the batch                                           */
   int64_t pairs_bound;         /* host-side count of ready pairs that triggered the launch      */
   float elapsed_ms;            /* device time first kernel -> last kernel; < 0 if not finished  */
+  float layout_ms;             /* histogram + scan + rank + scatter   (profile_kernels only,    */
+  float gemm1_ms;              /* gate/up GEMM with fused SiLU*up      else < 0)                 */
+  float gemm2_ms;              /* down GEMM                                                     */
+  float combine_ms;            /* weighted combine + unpermute                                  */
 } cep_invocation_info;
 
 /* Bytes of device workspace a plan with this configuration needs.  [host] out. */

@@ -32,13 +32,16 @@ class CepConfig(ctypes.Structure):
                 ("top_k", ctypes.c_int32), ("max_tokens", ctypes.c_int32), ("max_chunks", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("n_streams", ctypes.c_int32),
                 ("threshold_pairs", ctypes.c_int64), ("gemm_impl", ctypes.c_int32),
-                ("debug_checks", ctypes.c_int32)]
+                ("debug_checks", ctypes.c_int32), ("profile_kernels", ctypes.c_int32),
+                ("reserved_", ctypes.c_int32)]
 
 
 class InvocationInfo(ctypes.Structure):
     _fields_ = [("n_chunks", ctypes.c_int32), ("first_chunk_pos", ctypes.c_int32),
                 ("stream_index", ctypes.c_int32), ("n_tokens", ctypes.c_int32),
-                ("pairs_bound", ctypes.c_int64), ("elapsed_ms", ctypes.c_float)]
+                ("pairs_bound", ctypes.c_int64), ("elapsed_ms", ctypes.c_float),
+                ("layout_ms", ctypes.c_float), ("gemm1_ms", ctypes.c_float), ("gemm2_ms", ctypes.c_float),
+                ("combine_ms", ctypes.c_float)]
 
 
 class CepError(RuntimeError):
@@ -234,12 +237,12 @@ class MoELayer:
 
     def __init__(self, hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
                  dtype=CEP_BF16, mode=CEP_MODE_STREAMFFN, n_streams=2, threshold_pairs=0,
-                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, device="cuda"):
+                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, profile_kernels=0, device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the streamFFN library needs a CUDA device; there is no CPU path")
         self.cfg = CepConfig(hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
-                             dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks)
+                             dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks, profile_kernels, 0)
         self.device = torch.device(device)
         self.workspace = torch.empty(moe_plan_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
         self.packed = torch.empty(moe_packed_weight_bytes(self.cfg), dtype=torch.uint8, device=self.device)
