@@ -53,7 +53,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -153,7 +153,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="ep_shard")
@@ -300,7 +300,10 @@ def main():
     ffn_tflops = work["flops"] / ((g1_ms + g2_ms) * 1e-3) / 1e12
     g1_tflops = work["gemm1_flops"] / (g1_ms * 1e-3) / 1e12
     g2_tflops = work["gemm2_flops"] / (g2_ms * 1e-3) / 1e12
-    sustained = ms > 5.0          # a step of several ms runs under the power cap
+    # burst peak for a short timed region at full clocks, sustained peak once the run is long enough
+    # to sit under the power cap (clock well below maximum, or more than a second of back-to-back steps)
+    sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    sustained = (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
     peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     roofline = {"bound": "tensor", "kernel": "grouped_gemm_bf16_kernel<swiglu> (GEMM1: gate/up + SiLU*up)",
                 "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
