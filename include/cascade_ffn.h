@@ -220,6 +220,36 @@ CEP_API int moe_plan_destroy(cep_plan* plan);
 CEP_API const char* cep_last_error(const cep_plan* plan);
 
 /*
+ * layout_indices_noalloc: the integer half of the layout transform (per-expert counts, offsets,
+ * tile-aligned offsets, the stable row of every pair and the inverse map) for callers that cannot
+ * hand the library any scratch memory.  The paper has no counterpart: it exists for users who run
+ * inside a process whose memory pool already owns the device (an extra cudaMalloc would fail or eat
+ * into the KV cache) or who may not allocate on a latency-critical path.  It needs no plan and no
+ * workspace and calls no allocator: its scratch is a fixed array inside the library, about 1 MiB
+ * that every GPU loading the library holds until exit.
+ *   topk_ids        [device] int32 [n_tokens, top_k] global ids (one contiguous batch)
+ *   counts          [device] out int32 [E]
+ *   offsets         [device] out int32 [E+1]
+ *   padded_offsets  [device] out int32 [E+1]   group starts rounded up to CEP_ROW_ALIGN
+ *   row_of_pair     [device] out int32 [n_tokens*top_k]  tile-aligned row of each pair, -1 if not local
+ *   pair_of_row     [device] out int32 [pair_of_row_capacity]; entries of real rows are written,
+ *                   padding rows are left untouched; capacity >= padded_offsets[E]
+ *   status          [device] out int32 [2] or NULL: [0] != 0 an id was outside [0, n_experts_global),
+ *                   [1] != 0 a row did not fit pair_of_row_capacity
+ * Limits: n_experts_local <= 1024 and ceil(n_tokens*top_k / 2048) * n_experts_local <= 262144;
+ * larger requests return CEP_ERR_CAPACITY.  The work is enqueued on `stream`; outputs are ready when
+ * it completes.  The first call on each device looks up the array's device address (a blocking
+ * runtime query), so make that first call before any stream capture.  All calls share the one array,
+ * which keeps the previous call's contents (the part that must start at zero is cleared by every
+ * call): calls whose GPU work may overlap must be ordered by the caller or they race.
+ */
+CEP_API int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens, int32_t top_k,
+                                   int32_t n_experts_local, int32_t n_experts_global, int32_t* counts,
+                                   int32_t* offsets, int32_t* padded_offsets, int32_t* row_of_pair,
+                                   int32_t* pair_of_row, int32_t pair_of_row_capacity, int32_t* status,
+                                   void* stream);
+
+/*
  * Host-only helpers exported for CPU tests of the index arithmetic the kernels use.
  * cep_debug_decode_tile: maps a linear tile index to (expert, m_block, n_block) given the
  * per-expert m-tile prefix [E+1] and the number of n blocks; returns 0 or CEP_ERR_ARG.

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc"]
 
 
 class CepConfig(ctypes.Structure):
@@ -88,6 +88,7 @@ def load_library(build_if_missing: bool = True):
         "cep_last_error": (ctypes.c_char_p, [vp]),
         "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
         "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
+        "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -225,6 +226,18 @@ def cep_debug_schedule(pairs: Sequence[int], mode: int, theta: int) -> List[int]
     if n < 0:
         raise CepError(n, "cep_debug_schedule")
     return out[:len(pr)].tolist()
+
+
+def layout_indices_noalloc(topk_ids, n_experts_local: int, n_experts_global: int, counts, offsets,
+                           padded_offsets, row_of_pair, pair_of_row, status=None, stream=None) -> int:
+    """Index half of the layout transform with no workspace (all arguments are CUDA tensors the
+    caller allocated beforehand).  Returns the library's status code instead of raising, so a caller
+    can test the size limit."""
+    n_tokens, top_k = topk_ids.shape
+    return lib().layout_indices_noalloc(topk_ids.data_ptr(), n_tokens, top_k, n_experts_local, n_experts_global,
+                                        counts.data_ptr(), offsets.data_ptr(), padded_offsets.data_ptr(),
+                                        row_of_pair.data_ptr(), pair_of_row.data_ptr(), pair_of_row.numel(),
+                                        _dptr(status), _stream_handle(stream))
 
 
 # ---------------------------------------------------------------- convenience owner of the buffers

@@ -218,3 +218,82 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
 }
 
 }  // namespace cep
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the index part of the layout transform (histogram -> scan -> rank).
+//
+// Some users of this library cannot give it scratch memory at all: a plug-in running inside an
+// inference server whose memory pool already owns the whole device (a cudaMalloc there fails, or
+// steals from the KV cache), or a caller on a latency-critical path where an allocation would
+// synchronise the device.  For them the kernels' integer scratch (per-segment histograms, tile
+// prefix, status words) lives in the fixed array below, which every GPU that loads the library
+// holds (about 1 MiB) until the process exits.  The array is shared by all calls and keeps the
+// previous call's contents: what must start at zero is cleared at the start of each call, and
+// two calls whose GPU work overlaps (different streams, no ordering between them) race on it.
+namespace {
+
+constexpr int kNoAllocHistInts = 262144;          // room for n_segments * n_experts_local histogram cells
+constexpr int kNoAllocHeadInts = 2048;            // tile prefix [E+1 <= 1025] and the status words
+static __device__ __align__(256) int32_t g_noalloc_scratch[kNoAllocHeadInts + kNoAllocHistInts];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_noalloc_ptr[kMaxDevices] = {};         // device address of the array, per device
+
+// The array's name is only a host-side handle; its device address is looked up once per device.
+cudaError_t noalloc_scratch_address(int32_t** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_noalloc_ptr[dev]) {
+    int32_t* ptr = nullptr;
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens, int32_t top_k,
+                                      int32_t n_experts_local, int32_t n_experts_global, int32_t* counts,
+                                      int32_t* offsets, int32_t* padded_offsets, int32_t* row_of_pair,
+                                      int32_t* pair_of_row, int32_t pair_of_row_capacity, int32_t* status,
+                                      void* stream) {
+  using namespace cep;
+  if (!topk_ids || !counts || !offsets || !padded_offsets || !row_of_pair || !pair_of_row) return CEP_ERR_ARG;
+  if (n_tokens <= 0 || top_k <= 0 || top_k > 32 || n_experts_local <= 0 || n_experts_local > 1024 ||
+      n_experts_global < n_experts_local || pair_of_row_capacity <= 0)
+    return CEP_ERR_ARG;
+  const long long n_pairs = (long long)n_tokens * top_k;
+  if (n_pairs > (1ll << 30)) return CEP_ERR_CAPACITY;
+  const long long n_seg = (n_pairs + kSegPairs - 1) / kSegPairs;
+  if (n_seg * n_experts_local > kNoAllocHistInts) return CEP_ERR_CAPACITY;   // beyond the fixed scratch
+  int32_t* scratch = nullptr;
+  if (noalloc_scratch_address(&scratch) != cudaSuccess) return CEP_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t* tile_prefix = scratch;                       // [E+1]
+  int32_t* st_words = scratch + 1536;                   // [kStWords]
+  int32_t* seg_hist = scratch + kNoAllocHeadInts;       // [n_seg, E]
+  if (cudaMemsetAsync(st_words, 0, kStWords * sizeof(int32_t), st) != cudaSuccess) return CEP_ERR_CUDA;
+  BatchDesc batch{};
+  batch.chunk[0].ids = topk_ids;
+  batch.chunk[0].n_tokens = n_tokens;
+  batch.n_chunks = 1;
+  batch.n_tokens = n_tokens;
+  const int E = n_experts_local;
+  hist_kernel<<<(int)n_seg, kThreads, E * sizeof(int32_t), st>>>(batch, top_k, E, n_experts_global, seg_hist, st_words);
+  scan_kernel<<<1, 1024, 0, st>>>((int)n_seg, E, seg_hist, counts, offsets, padded_offsets, tile_prefix);
+  rank_kernel<<<(int)n_seg, kThreads, kWarps * E * sizeof(int32_t), st>>>(batch, top_k, E, seg_hist, row_of_pair,
+                                                                        pair_of_row, pair_of_row_capacity, st_words);
+  if (cudaGetLastError() != cudaSuccess) return CEP_ERR_CUDA;
+  if (status) {
+    // status[0]: an id was outside [0, n_experts_global); status[1]: a row did not fit pair_of_row
+    if (cudaMemcpyAsync(status, st_words + kStBadRouting, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(status + 1, st_words + kStBoundsViolation, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return CEP_ERR_CUDA;
+  }
+  return CEP_OK;
+}
