@@ -159,6 +159,7 @@ def main():
     ap.add_argument("--config", default="ep_shard")
     ap.add_argument("--streams", type=int, default=2)
     ap.add_argument("--oracle-tokens", type=int, default=48)
+    ap.add_argument("--gemm-impl", type=int, default=0, help="0: CTA-pair tcgen05 (product), 2: one-CTA tcgen05")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -195,7 +196,8 @@ def main():
     ch_pairs = [int((inp.topk_ids[o:o + n] < cfg.E_local).sum().item()) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
 
     layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks,
-                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, profile_kernels=1)
+                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, profile_kernels=1,
+                         gemm_impl=args.gemm_impl)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     torch.cuda.synchronize()
     out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")

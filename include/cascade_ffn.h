@@ -81,8 +81,10 @@ typedef enum {
 } cep_mode;
 
 typedef enum {
-  CEP_GEMM_TCGEN05 = 0,        /* tcgen05/TMEM tiles fed by TMA (the product path)              */
-  CEP_GEMM_SIMT = 1            /* slow CUDA-core kernel, kept for fault isolation in tests      */
+  CEP_GEMM_TCGEN05 = 0,        /* tcgen05/TMEM tiles fed by TMA, CTA pairs on 256x256 tiles
+                                  (the product path)                                            */
+  CEP_GEMM_SIMT = 1,           /* slow CUDA-core kernel, kept for fault isolation in tests      */
+  CEP_GEMM_TCGEN05_1CTA = 2    /* tcgen05 with one CTA per 128x256 tile (comparison variant)    */
 } cep_gemm_impl;
 
 #define CEP_MAX_CHUNKS_PER_INVOCATION 32   /* a batch is launched early when it holds this many */
@@ -252,12 +254,14 @@ CEP_API int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens, in
 /*
  * Host-only helpers exported for CPU tests of the index arithmetic the kernels use.
  * cep_debug_decode_tile: maps a linear tile index to (expert, m_block, n_block) given the
- * per-expert m-tile prefix [E+1] and the number of n blocks; returns 0 or CEP_ERR_ARG.
+ * per-expert m-tile prefix [E+1], the number of n blocks and the n blocks per L2-resident chunk;
+ * returns 0 or CEP_ERR_ARG.
  * cep_debug_schedule: replays the host scheduler on a list of per-chunk pair counts and
  * writes, per chunk position, the invocation it lands in; returns the invocation count.
  */
 CEP_API int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n,
-                          int32_t tile, int32_t* expert, int32_t* m_block, int32_t* n_block);
+                          int32_t n_group, int32_t tile, int32_t* expert, int32_t* m_block,
+                          int32_t* n_block);
 CEP_API int cep_debug_schedule(const int64_t* pairs, int32_t n_chunks, int32_t mode, int64_t theta,
                        int32_t* invocation_of_chunk);
 

@@ -11,4 +11,4 @@ from .binding import (CepConfig, CepError, InvocationInfo, MoELayer, lib, load_l
                       ffn_query, ffn_debug_export, cep_kernel_launches, moe_plan_destroy, cep_last_error,
                       cep_debug_decode_tile, cep_debug_schedule, layout_indices_noalloc,
                       CEP_BF16, CEP_FP8_E4M3_BLOCK128, CEP_MODE_SYNC, CEP_MODE_ASYNC, CEP_MODE_STREAMFFN,
-                      CEP_GEMM_TCGEN05, CEP_GEMM_SIMT, STATUS_NAMES)
+                      CEP_GEMM_TCGEN05, CEP_GEMM_SIMT, CEP_GEMM_TCGEN05_1CTA, STATUS_NAMES)

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libcascade_ffn.so")
 
 CEP_BF16, CEP_FP8_E4M3_BLOCK128 = 0, 1
 CEP_MODE_SYNC, CEP_MODE_ASYNC, CEP_MODE_STREAMFFN = 0, 1, 2
-CEP_GEMM_TCGEN05, CEP_GEMM_SIMT = 0, 1
+CEP_GEMM_TCGEN05, CEP_GEMM_SIMT, CEP_GEMM_TCGEN05_1CTA = 0, 1, 2
 STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ERR_WORKSPACE",
                 -4: "CEP_ERR_CAPACITY", -5: "CEP_ERR_INCOMPLETE", -6: "CEP_ERR_BAD_ROUTING",
                 -7: "CEP_ERR_DEVICE_TIMEOUT", -8: "CEP_ERR_CUDA", -9: "CEP_ERR_UNSUPPORTED"}
@@ -86,7 +86,7 @@ def load_library(build_if_missing: bool = True):
         "cep_kernel_launches": (i64, [vp]),
         "moe_plan_destroy": (ctypes.c_int, [vp]),
         "cep_last_error": (ctypes.c_char_p, [vp]),
-        "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
+        "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
         "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
@@ -208,11 +208,12 @@ def cep_last_error(plan=None) -> str:
     return m.decode() if m else ""
 
 
-def cep_debug_decode_tile(tile_prefix, n_blocks_n: int, tile: int):
+def cep_debug_decode_tile(tile_prefix, n_blocks_n: int, tile: int, n_group: int = 0):
     import numpy as np
     tp = np.ascontiguousarray(tile_prefix, dtype=np.int32)
     e, m, n = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
-    rc = lib().cep_debug_decode_tile(tp.ctypes.data_as(ctypes.c_void_p), tp.shape[0] - 1, n_blocks_n, tile,
+    rc = lib().cep_debug_decode_tile(tp.ctypes.data_as(ctypes.c_void_p), tp.shape[0] - 1, n_blocks_n,
+                                     n_group if n_group > 0 else n_blocks_n, tile,
                                      ctypes.byref(e), ctypes.byref(m), ctypes.byref(n))
     return None if rc else (e.value, m.value, n.value)
 

@@ -10,7 +10,6 @@ namespace cep {
 constexpr int kRowAlign = CEP_ROW_ALIGN;        // rows per GEMM M tile; expert groups start on multiples
 constexpr int kMaxChunksPerInv = CEP_MAX_CHUNKS_PER_INVOCATION;
 constexpr int kSegPairs = 2048;                 // pairs per block in the histogram / rank kernels
-constexpr int kGroupM = 16;                     // m-tiles per scheduling group (L2 reuse of A rows)
 constexpr int kQuantBlock = 128;                // fp8 scale block
 
 // Device status word layout (int32 each).
@@ -44,18 +43,20 @@ struct LayoutPtrs {
   int32_t* row_of_pair;       // [max_tokens*k] physical row, -1 when not local
   int32_t* pair_of_row;       // [cap_rows] batch pair index, -1 on padding
   int32_t* status;            // [kStWords]
+  int32_t* sched;             // [2] tile counters of the two GEMMs of an invocation (zeroed by the scan kernel)
 };
 
 // ---------------------------------------------------------------- tile scheduling arithmetic
-// Linear tile index -> (expert, m_block, n_block).  Tiles are expert-major; inside an
-// expert, m-tiles are taken in groups of kGroupM, and inside a group the n block is the
-// slow index, so that concurrently running CTAs share one weight tile and a group's
-// activation rows stay L2-resident while the expert's weights stream past them.
+// Linear tile index -> (expert, m_block, n_block).  Tiles are expert-major.  Inside an expert the n
+// blocks are taken in chunks of `n_group` (the last chunk may be shorter); a chunk is swept over all
+// m blocks of the expert with n as the fast index.  The CTAs running at one time then share the
+// chunk's weight panel (sized by the caller to stay L2-resident for the whole sweep) while the
+// expert's activation rows stream past it, one pass per chunk.
 struct TileCoord { int expert, m_block, n_block; };
 
 __host__ __device__ inline bool decode_tile(const int32_t* __restrict__ tile_prefix, int n_experts,
-                                            int n_blocks_n, int tile, TileCoord* out) {
-  if (tile < 0 || n_blocks_n <= 0) return false;
+                                            int n_blocks_n, int n_group, int tile, TileCoord* out) {
+  if (tile < 0 || n_blocks_n <= 0 || n_group <= 0) return false;
   int lo = 0, hi = n_experts;            // find e: prefix[e]*NB <= tile < prefix[e+1]*NB
   if ((long long)tile >= (long long)tile_prefix[n_experts] * n_blocks_n) return false;
   while (hi - lo > 1) {
@@ -65,15 +66,24 @@ __host__ __device__ inline bool decode_tile(const int32_t* __restrict__ tile_pre
   // now prefix[lo] <= tile / NB < prefix[lo+1]: expert lo has tiles and owns this one
   const int mt = tile_prefix[lo + 1] - tile_prefix[lo];
   const int li = tile - tile_prefix[lo] * n_blocks_n;
-  const int per_group = kGroupM * n_blocks_n;
-  const int g = li / per_group;
-  const int rem = li - g * per_group;
-  int gm = mt - g * kGroupM;
-  if (gm > kGroupM) gm = kGroupM;
+  const int c = li / (mt * n_group);                 // chunk of n blocks (all but the last are full)
+  const int rem = li - c * mt * n_group;
+  int gn = n_blocks_n - c * n_group;
+  if (gn > n_group) gn = n_group;
   out->expert = lo;
-  out->n_block = rem / gm;
-  out->m_block = g * kGroupM + rem % gm;
+  out->m_block = rem / gn;
+  out->n_block = c * n_group + (rem - out->m_block * gn);
   return true;
+}
+
+// n blocks per chunk so that one chunk's weight panel (block_cols x K elements each) stays within a
+// budget the L2 keeps resident next to the streamed operand.
+__host__ inline int n_group_for(int n_blocks_n, int block_cols, int K, int elt_bytes) {
+  const long long budget = 32ll << 20;
+  long long g = budget / ((long long)block_cols * K * elt_bytes);
+  if (g < 1) g = 1;
+  if (g > n_blocks_n) g = n_blocks_n;
+  return (int)g;
 }
 
 // ---------------------------------------------------------------- kernel launchers (defined in the .cu files)

@@ -16,6 +16,7 @@
 
 #include "cep_common.h"
 #include "gemm_tcgen05.h"
+#include "tcgen05_ptx.cuh"
 
 namespace cep {
 namespace {
@@ -29,7 +30,6 @@ constexpr int B_STAGE = BN * BKB;       // 32 KiB
 constexpr int kThreads = 192;
 constexpr int kEpiWarp0 = 2;
 constexpr int kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct __align__(8) Barriers {
   uint64_t full[kStages], empty[kStages], acc_full[2], acc_empty[2];
@@ -39,99 +39,72 @@ struct __align__(8) Barriers {
 constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE) + 1024 /*alignment slack*/ + 256;
 static_assert(sizeof(Barriers) <= 256, "barrier block");
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the wait was abandoned (this or another role timed out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer();
-  for (uint32_t spin = 1;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 1023u) == 0u) {
-      if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(&status[kStTimeout], 1);
-        return false;
+using namespace ptx;
+
+// Epilogue of one 128-row x 256-column accumulator: each thread owns one row (one tensor-memory
+// lane), reads it 32 columns at a time, applies SiLU(gate)*up when the tile holds [128 gate | 128 up]
+// columns, rounds to bf16 once and stores 64 contiguous bytes.  Rows at or beyond the expert's
+// count (padding, or the next expert's rows under a pair tile) are not stored.
+template <bool kSwiglu>
+__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, int r_in_group, int expert, int n_block,
+                                              int n_out_cols, int out_ld, __nv_bfloat16* __restrict__ out,
+                                              const int32_t* __restrict__ counts,
+                                              const int32_t* __restrict__ padded_offsets) {
+  const bool row_ok = r_in_group < counts[expert];
+  const size_t grow = (size_t)(padded_offsets[expert] + r_in_group);
+  if (kSwiglu) {
+    __nv_bfloat16* orow = out + grow * out_ld + n_block * (BN / 2);
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t g[32], u[32];
+      tc_ld32(t_addr + c * 32, g);
+      tc_ld32(t_addr + 128 + c * 32, u);
+      tc_wait_ld();
+      if (row_ok && n_block * (BN / 2) + c * 32 < n_out_cols) {
+        uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint4 v;
+          v.x = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 0]), __uint_as_float(u[8 * q + 0])),
+                          silu_mul(__uint_as_float(g[8 * q + 1]), __uint_as_float(u[8 * q + 1])));
+          v.y = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 2]), __uint_as_float(u[8 * q + 2])),
+                          silu_mul(__uint_as_float(g[8 * q + 3]), __uint_as_float(u[8 * q + 3])));
+          v.z = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 4]), __uint_as_float(u[8 * q + 4])),
+                          silu_mul(__uint_as_float(g[8 * q + 5]), __uint_as_float(u[8 * q + 5])));
+          v.w = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 6]), __uint_as_float(u[8 * q + 6])),
+                          silu_mul(__uint_as_float(g[8 * q + 7]), __uint_as_float(u[8 * q + 7])));
+          dst[q] = v;
+        }
+      }
+    }
+  } else {
+    __nv_bfloat16* orow = out + grow * out_ld + n_block * BN;
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+      uint32_t d[32];
+      tc_ld32(t_addr + c * 32, d);
+      tc_wait_ld();
+      if (row_ok && n_block * BN + c * 32 < n_out_cols) {
+        uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(d[8 * q + 0]), __uint_as_float(d[8 * q + 1]));
+          v.y = pack_bf16(__uint_as_float(d[8 * q + 2]), __uint_as_float(d[8 * q + 3]));
+          v.z = pack_bf16(__uint_as_float(d[8 * q + 4]), __uint_as_float(d[8 * q + 5]));
+          v.w = pack_bf16(__uint_as_float(d[8 * q + 6]), __uint_as_float(d[8 * q + 7]));
+          dst[q] = v;
+        }
       }
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
-  d |= (uint64_t)1 << 46;                            // descriptor version (sm_100)
-  d |= (uint64_t)2 << 61;                            // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor for kind::f16: fp32 accumulate, bf16 x bf16, both K-major, M=128, N=256.
-__host__ __device__ constexpr uint32_t make_idesc_bf16() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-__device__ __forceinline__ float silu_mul(float g, float u) { return (g / (1.f + __expf(-g))) * u; }
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
-
-// ------------------------------------------------------------------ the kernel
+// ------------------------------------------------------------------ the kernel (one CTA per tile)
 template <bool kSwiglu>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                         int num_kb /*K*2/128*/, int n_blocks_n, int n_experts, int n_out_cols, int out_ld,
+                         int num_kb /*K*2/128*/, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
                          __nv_bfloat16* __restrict__ out, const int32_t* __restrict__ tile_prefix,
                          const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
                          int32_t* __restrict__ status) {
@@ -167,7 +140,7 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         TileCoord tc;
-        if (!decode_tile(tile_prefix, n_experts, n_blocks_n, tile, &tc)) break;
+        if (!decode_tile(tile_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
         const int row0 = padded_offsets[tc.expert] + tc.m_block * BM;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
@@ -182,7 +155,7 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16();
+      constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
@@ -212,59 +185,12 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       TileCoord tc;
-      if (!decode_tile(tile_prefix, n_experts, n_blocks_n, tile, &tc)) break;
+      if (!decode_tile(tile_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
       if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status)) break;
       tc_fence_after();
-      const int r_in_group = tc.m_block * BM + lane_grp * 32 + lane;
-      const bool row_ok = r_in_group < counts[tc.expert];
-      const size_t grow = (size_t)(padded_offsets[tc.expert] + r_in_group);
-      const uint32_t t_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN);
-      if (kSwiglu) {
-        __nv_bfloat16* orow = out + grow * out_ld + tc.n_block * (BN / 2);
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t g[32], u[32];
-          tc_ld32(t_addr + c * 32, g);
-          tc_ld32(t_addr + 128 + c * 32, u);
-          tc_wait_ld();
-          if (row_ok && tc.n_block * (BN / 2) + c * 32 < n_out_cols) {
-            uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint4 v;
-              v.x = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 0]), __uint_as_float(u[8 * q + 0])),
-                              silu_mul(__uint_as_float(g[8 * q + 1]), __uint_as_float(u[8 * q + 1])));
-              v.y = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 2]), __uint_as_float(u[8 * q + 2])),
-                              silu_mul(__uint_as_float(g[8 * q + 3]), __uint_as_float(u[8 * q + 3])));
-              v.z = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 4]), __uint_as_float(u[8 * q + 4])),
-                              silu_mul(__uint_as_float(g[8 * q + 5]), __uint_as_float(u[8 * q + 5])));
-              v.w = pack_bf16(silu_mul(__uint_as_float(g[8 * q + 6]), __uint_as_float(u[8 * q + 6])),
-                              silu_mul(__uint_as_float(g[8 * q + 7]), __uint_as_float(u[8 * q + 7])));
-              dst[q] = v;
-            }
-          }
-        }
-      } else {
-        __nv_bfloat16* orow = out + grow * out_ld + tc.n_block * BN;
-#pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-          uint32_t d[32];
-          tc_ld32(t_addr + c * 32, d);
-          tc_wait_ld();
-          if (row_ok && tc.n_block * BN + c * 32 < n_out_cols) {
-            uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint4 v;
-              v.x = pack_bf16(__uint_as_float(d[8 * q + 0]), __uint_as_float(d[8 * q + 1]));
-              v.y = pack_bf16(__uint_as_float(d[8 * q + 2]), __uint_as_float(d[8 * q + 3]));
-              v.z = pack_bf16(__uint_as_float(d[8 * q + 4]), __uint_as_float(d[8 * q + 5]));
-              v.w = pack_bf16(__uint_as_float(d[8 * q + 6]), __uint_as_float(d[8 * q + 7]));
-              dst[q] = v;
-            }
-          }
-        }
-      }
+      epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
+                             tc.m_block * BM + lane_grp * 32 + lane, tc.expert, tc.n_block, n_out_cols, out_ld, out,
+                             counts, padded_offsets);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[acc]));
@@ -272,12 +198,243 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
     }
   }
   // ------------------------------------------------------------------ teardown
+#ifdef CEP_EXP_TIMESTAMPS
+  if (threadIdx.x == 64) status[8 + blockIdx.x] = (int32_t)(globaltimer() >> 8);     // 256 ns units
+#endif
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+
+// ------------------------------------------------------------------ the kernel (a CTA pair per 256x256 tile)
+// Two CTAs of a cluster share one tile of 256 rows x 256 accumulator columns (tcgen05 cta_group::2):
+// each loads its own 128 activation rows and HALF of the weight tile, the leader (cluster rank 0)
+// issues M=256 MMAs that read both CTAs' shared memory, and each CTA keeps the accumulator of its
+// own 128 rows in its own tensor memory.  Per k-step an SM takes in 32 KB instead of 48 KB for the
+// same number of MMA cycles.  An expert with an odd number of 128-row blocks leaves the second half
+// of its last pair tile empty (those rows are computed and not stored).
+//
+// Barriers: full[s] (leader; its producer's arrival + both CTAs' TMA bytes), empty[s] (one per CTA,
+// arrived by the leader's commit), acc_full[a] (one per CTA, leader's commit), acc_empty[a] (leader;
+// 4 epilogue warps x 2 CTAs).
+#ifndef CEP_PAIR_STAGES
+#define CEP_PAIR_STAGES 6
+#endif
+constexpr int kPairStages = CEP_PAIR_STAGES;
+constexpr int PB_STAGE = (BN / 2) * BKB;               // 16 KiB: this CTA's half of the weight tile
+constexpr int kMaxExperts = 1024;
+constexpr int kSchedRing = 4;                          // tile ids in flight between the scheduler and its readers
+constexpr int kSchedReaders = 11;                      // leader: producer, MMA, 4 epilogue warps; peer: producer, 4 epilogue warps
+constexpr int kPairThreads = 224;                      // warp 6 of the leader CTA hands out tiles
+struct __align__(8) PairBarriers {
+  uint64_t full[kPairStages], empty[kPairStages], acc_full[2], acc_empty[2];
+  uint64_t sched_full[kSchedRing], sched_empty[kSchedRing];
+  int32_t sched_tile[kSchedRing];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// Reader side of the tile ring: every reading role (a single thread, or a warp in lock-step) walks
+// the ring in order; -1 ends the kernel.  The peer CTA's copy of the ring is written by the leader
+// through the cluster, so its readers acquire at cluster scope.
+struct TileReader {
+  int slot = 0; uint32_t phase = 0;
+  // Waits for the next tile id.  The caller must call done() once every thread of the role has the value.
+  __device__ __forceinline__ int next(PairBarriers* bars, bool is_peer, volatile int* abort_flag, int32_t* status) {
+    const uint32_t bar = smem_u32(&bars->sched_full[slot]);
+    const bool ok = is_peer ? mbar_wait_acq_cluster(bar, phase, abort_flag, status) : mbar_wait(bar, phase, abort_flag, status);
+    if (!ok) return -1;
+    return bars->sched_tile[slot];
+  }
+  // Frees the ring slot for the scheduler (one arrival per reading role) and advances.
+  __device__ __forceinline__ void done(PairBarriers* bars, bool signal) {
+    if (signal) mbar_arrive_cluster(mapa(smem_u32(&bars->sched_empty[slot]), 0));
+    if (++slot == kSchedRing) { slot = 0; phase ^= 1u; }
+  }
+};
+constexpr int kPairSmemBytes = kPairStages * (A_STAGE + PB_STAGE) + (kMaxExperts + 1) * 4 + 1024 + 256;
+static_assert(sizeof(PairBarriers) <= 256, "barrier block");
+
+template <bool kSwiglu>
+__global__ void __launch_bounds__(kPairThreads, 1)
+grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                              int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
+                              __nv_bfloat16* __restrict__ out, const int32_t* __restrict__ tile_prefix,
+                              const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
+                              int32_t* __restrict__ tile_counter, int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + kPairStages * A_STAGE;
+  PairBarriers* bars = reinterpret_cast<PairBarriers*>(smem + kPairStages * (A_STAGE + PB_STAGE));
+  int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kPairStages * (A_STAGE + PB_STAGE) + 256);   // [E+1]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  volatile int* abort_flag = &bars->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), 8); }
+    for (int s = 0; s < kSchedRing; ++s) { mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders); }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x == 32) {          // cumulative number of pair tiles (two 128-row blocks) per expert
+    int run = 0;
+    for (int e = 0; e < n_experts; ++e) {
+      pair_prefix[e] = run;
+      run += (tile_prefix[e + 1] - tile_prefix[e] + 1) >> 1;
+    }
+    pair_prefix[n_experts] = run;
+  }
+  __syncthreads();
+  if (warp == 1) {                  // executed by the same warp of both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();               // both CTAs' barriers are initialised before any remote arrival
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  const int total_tiles = pair_prefix[n_experts] * n_blocks_n;
+  const bool is_peer = rank != 0;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      TileReader rd;
+      for (;ok;) {
+        const int tile = rd.next(bars, is_peer, abort_flag, status);
+        rd.done(bars, true);
+        if (tile < 0) break;
+        TileCoord tc;
+        if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
+        const int row0 = padded_offsets[tc.expert] + tc.m_block * (2 * BM) + (int)rank * BM;
+        const int n0 = tc.n_block * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < num_kb; ++kb) {
+#ifdef CEP_EXP_NO_LOAD
+          ok = false; break;
+#endif
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);        // the leader's barrier
+          // the leader alone arrives, announcing both CTAs' bytes; the peer's bytes can only land in
+          // this phase because its loads wait for the stage to be freed by the leader's MMAs
+          if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), 2 * (A_STAGE + PB_STAGE));
+          tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * (BKB / 2), row0, full);
+          tma_load_3d_pair(smem_u32(smem_b + stage * PB_STAGE), &tm_b, kb * (BKB / 2), n0, tc.expert, full);
+          if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(2 * BM, BN);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      TileReader rd;
+      for (;ok;) {
+        const int tile = rd.next(bars, false, abort_flag, status);
+        rd.done(bars, true);
+        if (tile < 0) break;
+        if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+#ifndef CEP_EXP_NO_LOAD
+          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status)) { ok = false; break; }
+#endif
+          tc_fence_after();
+          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE));
+          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * PB_STAGE));
+#ifndef CEP_EXP_NO_MMA
+#pragma unroll
+          for (int k4 = 0; k4 < BKB / 32; ++k4)
+            tc_mma_f16_pair(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0 ? 1u : 0u);
+#endif
+#ifdef CEP_PAIR_TWO_COMMITS
+          const uint32_t e_bar = smem_u32(&bars->empty[stage]);
+          tc_commit_pair(mapa(e_bar, 0));               // frees the stage in both CTAs
+          tc_commit_pair(mapa(e_bar, 1));
+#else
+          tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);   // frees the stage in both CTAs
+#endif
+          if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+#ifdef CEP_PAIR_TWO_COMMITS
+        const uint32_t f_bar = smem_u32(&bars->acc_full[acc]);
+        tc_commit_pair(mapa(f_bar, 0));                 // accumulator complete, both halves
+        tc_commit_pair(mapa(f_bar, 1));
+#else
+        tc_commit_pair_both(smem_u32(&bars->acc_full[acc]), 3);  // accumulator complete, both halves
+#endif
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp == 6) {
+    // ---------------------------------------------------------------- tile scheduler (leader CTA only)
+    // Tiles are handed out in linear order from a global counter, so the CTA pairs running at any time
+    // work on neighbouring tiles whatever their individual speeds: the set of operand rows in flight
+    // (and so the L2 working set) stays one wave wide instead of spreading as slower pairs fall behind.
+    if (lane == 0 && !is_peer) {
+      int slot = 0; uint32_t phase = 0;
+      for (;;) {
+        if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1u, abort_flag, status)) break;
+        int t = atomicAdd(tile_counter, 1);
+        if (t >= total_tiles) t = -1;
+        bars->sched_tile[slot] = t;
+        st_shared_cluster_u32(mapa(smem_u32(&bars->sched_tile[slot]), 1), (uint32_t)t);
+        mbar_arrive(smem_u32(&bars->sched_full[slot]));
+        mbar_arrive_release_cluster(mapa(smem_u32(&bars->sched_full[slot]), 1));
+        if (t < 0) break;
+        if (++slot == kSchedRing) { slot = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5, both CTAs)
+    const int lane_grp = warp & 3;
+    int acc = 0; uint32_t acc_phase = 0;
+    TileReader rd;
+    for (;;) {
+      const int tile = rd.next(bars, is_peer, abort_flag, status);
+      __syncwarp();                                    // every lane holds the id before the slot is freed
+      rd.done(bars, lane == 0);
+      if (tile < 0) break;
+      TileCoord tc;
+      if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
+      if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status)) break;
+      tc_fence_after();
+      epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
+                             tc.m_block * (2 * BM) + (int)rank * BM + lane_grp * 32 + lane, tc.expert, tc.n_block,
+                             n_out_cols, out_ld, out, counts, padded_offsets);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&bars->acc_empty[acc]), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+#ifdef CEP_EXP_TIMESTAMPS
+  if (threadIdx.x == 64) status[8 + blockIdx.x] = (int32_t)(globaltimer() >> 8);     // 256 ns units
+#endif
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();               // no CTA leaves while its peer may still signal or read it
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -322,6 +479,63 @@ int make_operand_map(GemmTensorMap* out, const void* base, int elt_bytes, int K,
 int gemm_tile_rows() { return BM; }
 int gemm_tile_cols() { return BN; }
 
+static int g_pair_clusters = -1;      // co-resident CTA pairs on this device (0: pairs unavailable)
+
+static cudaError_t setup_pair_kernels(int n_sms) {
+  if (g_pair_clusters >= 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(n_sms & ~1, 1, 1); cfg.blockDim = dim3(kPairThreads, 1, 1);
+  cfg.dynamicSmemBytes = kPairSmemBytes; cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = 0;
+  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_bf16_pair_kernel<true>, &cfg);
+  if (e != cudaSuccess) return e;
+  g_pair_clusters = n;
+  return cudaSuccess;
+}
+
+int gemm_pair_clusters() { return g_pair_clusters; }
+
+cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                                     void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
+                                     int64_t* launches) {
+  if (p.is_fp8) return cudaErrorNotSupported;
+  cudaError_t e = setup_pair_kernels(n_sms);
+  if (e != cudaSuccess) return e;
+  if (g_pair_clusters < 1) return cudaErrorNotSupported;
+  const int n_blocks_n = (p.N + BN - 1) / BN;
+  const int n_out_cols = p.swiglu ? p.N / 2 : p.N;
+  int clusters = max_pair_tiles < g_pair_clusters ? max_pair_tiles : g_pair_clusters;
+  if (clusters < 1) return cudaSuccess;
+  int num_kb = p.K * 2 / BKB;
+  int n_experts = p.n_experts, out_ld = p.out_ld;
+  int n_group = n_group_for(n_blocks_n, BN, p.K, 2);
+  int32_t* counter = lp.sched + (p.swiglu ? 0 : 1);     // zeroed by this invocation's scan kernel
+  __nv_bfloat16* o = (__nv_bfloat16*)out;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(2 * clusters, 1, 1); cfg.blockDim = dim3(kPairThreads, 1, 1);
+  cfg.dynamicSmemBytes = kPairSmemBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+  const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
+  const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
+  if (p.swiglu)
+    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<true>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
+                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, counter, lp.status);
+  else
+    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<false>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
+                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, counter, lp.status);
+  *launches += 1;
+  return e;
+}
+
 cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                                 void* out, const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s,
                                 int64_t* launches) {
@@ -339,13 +553,14 @@ cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a,
   int grid = max_tiles < n_sms ? max_tiles : n_sms;
   if (grid < 1) return cudaSuccess;
   const int num_kb = p.K * 2 / BKB;
+  const int n_group = n_group_for(n_blocks_n, BN, p.K, 2);
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
   if (p.swiglu)
-    grouped_gemm_bf16_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(a, b, num_kb, n_blocks_n, p.n_experts, n_out_cols,
+    grouped_gemm_bf16_kernel<true><<<grid, kThreads, kSmemBytes, s>>>(a, b, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols,
         p.out_ld, (__nv_bfloat16*)out, lp.tile_prefix, lp.counts, lp.padded_offsets, lp.status);
   else
-    grouped_gemm_bf16_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(a, b, num_kb, n_blocks_n, p.n_experts, n_out_cols,
+    grouped_gemm_bf16_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(a, b, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols,
         p.out_ld, (__nv_bfloat16*)out, lp.tile_prefix, lp.counts, lp.padded_offsets, lp.status);
   *launches += 1;
   return cudaGetLastError();

@@ -19,4 +19,11 @@ cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a,
                                 void* out, const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s,
                                 int64_t* launches);
 
+// CTA-pair variant (256-row x 256-column tiles, tcgen05 cta_group::2).  box_rows of its weight operand
+// map is gemm_tile_cols()/2.  max_pair_tiles bounds the number of pair tiles (for the grid size).
+cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                                     void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
+                                     int64_t* launches);
+int gemm_pair_clusters();
+
 }  // namespace cep

@@ -48,8 +48,9 @@ hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global,
 __global__ void __launch_bounds__(1024)
 scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: row base*/,
             int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ padded_offsets,
-            int32_t* __restrict__ tile_prefix) {
+            int32_t* __restrict__ tile_prefix, int32_t* __restrict__ sched) {
   __shared__ int32_t s_cnt[1024];
+  if (threadIdx.x < 2) sched[threadIdx.x] = 0;   // tile counters of this invocation's two GEMMs
   __shared__ int32_t s_off[1025], s_pad[1025];
   const int e = threadIdx.x;
   int total = 0;
@@ -204,7 +205,7 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
   hist_kernel<<<n_seg, kThreads, E * sizeof(int32_t), s>>>(batch, k, E, cfg.n_experts_global, lp.block_base,
                                                            lp.status);
   scan_kernel<<<1, 1024, 0, s>>>(n_seg, E, lp.block_base, lp.counts, lp.offsets, lp.padded_offsets,
-                                 lp.tile_prefix);
+                                 lp.tile_prefix, lp.sched);
   rank_kernel<<<n_seg, kThreads, kWarps * E * sizeof(int32_t), s>>>(batch, k, E, lp.block_base, lp.row_of_pair,
                                                                    lp.pair_of_row, cap_rows, lp.status);
   const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128;
@@ -285,7 +286,7 @@ extern "C" int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens,
   batch.n_tokens = n_tokens;
   const int E = n_experts_local;
   hist_kernel<<<(int)n_seg, kThreads, E * sizeof(int32_t), st>>>(batch, top_k, E, n_experts_global, seg_hist, st_words);
-  scan_kernel<<<1, 1024, 0, st>>>((int)n_seg, E, seg_hist, counts, offsets, padded_offsets, tile_prefix);
+  scan_kernel<<<1, 1024, 0, st>>>((int)n_seg, E, seg_hist, counts, offsets, padded_offsets, tile_prefix, scratch + 1600);
   rank_kernel<<<(int)n_seg, kThreads, kWarps * E * sizeof(int32_t), st>>>(batch, top_k, E, seg_hist, row_of_pair,
                                                                         pair_of_row, pair_of_row_capacity, st_words);
   if (cudaGetLastError() != cudaSuccess) return CEP_ERR_CUDA;

@@ -53,7 +53,7 @@ bool should_launch(int mode, int64_t pending_pairs, int pending_chunks, int64_t 
 struct Layout {                                   // byte offsets inside the workspace
   size_t status;
   size_t slot0, slot_bytes;
-  size_t counts, offsets, padded, tile_prefix, block_base, row_of_pair, pair_of_row, xp, xp_scales, act,
+  size_t counts, offsets, padded, tile_prefix, sched, block_base, row_of_pair, pair_of_row, xp, xp_scales, act,
       act_scales, y;                              // offsets inside a slot
   size_t total;
   int cap_rows, n_seg_max;
@@ -73,7 +73,7 @@ int validate(const cep_config* c, const char** why) {
   if (c->mode < CEP_MODE_SYNC || c->mode > CEP_MODE_STREAMFFN) { *why = "unknown mode"; return CEP_ERR_ARG; }
   if (c->n_streams < 1 || c->n_streams > 16) { *why = "n_streams must be in 1..16"; return CEP_ERR_ARG; }
   if (c->threshold_pairs < 0) { *why = "threshold_pairs must be >= 0"; return CEP_ERR_ARG; }
-  if (c->gemm_impl != CEP_GEMM_TCGEN05 && c->gemm_impl != CEP_GEMM_SIMT) { *why = "unknown gemm_impl"; return CEP_ERR_ARG; }
+  if (c->gemm_impl < CEP_GEMM_TCGEN05 || c->gemm_impl > CEP_GEMM_TCGEN05_1CTA) { *why = "unknown gemm_impl"; return CEP_ERR_ARG; }
   return CEP_OK;
 }
 
@@ -92,6 +92,7 @@ Layout make_layout(const cep_config& c) {
   L.offsets = o; o = align_up(o + (E + 1) * 4, A);
   L.padded = o; o = align_up(o + (E + 1) * 4, A);
   L.tile_prefix = o; o = align_up(o + (E + 1) * 4, A);
+  L.sched = o; o = align_up(o + 2 * 4, A);
   L.block_base = o; o = align_up(o + (size_t)L.n_seg_max * E * 4, A);
   L.row_of_pair = o; o = align_up(o + (size_t)max_pairs * 4, A);
   L.pair_of_row = o; o = align_up(o + (size_t)L.cap_rows * 4, A);
@@ -198,6 +199,15 @@ int launch_invocation(cep_plan* p) {
       CUDA_TRY(p, launch_gemm_simt(g1, sl.xp, p->w13p, sl.act, sl.lp, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
       CUDA_TRY(p, launch_gemm_simt(g2, sl.act, p->w2p, sl.y, sl.lp, st, &p->launches));
+    } else if (c.gemm_impl == CEP_GEMM_TCGEN05) {
+      const int bn = gemm_tile_cols();
+      const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
+      const long long t1 = pair_bound * ((g1.N + bn - 1) / bn), t2 = pair_bound * ((g2.N + bn - 1) / bn);
+      CUDA_TRY(p, launch_gemm_tcgen05_pair(g1, sl.tm_a1, p->tm_b1, sl.act, sl.lp, (int)(t1 > (1 << 30) ? (1 << 30) : t1),
+                                           p->n_sms, st, &p->launches));
+      if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
+      CUDA_TRY(p, launch_gemm_tcgen05_pair(g2, sl.tm_a2, p->tm_b2, sl.y, sl.lp, (int)(t2 > (1 << 30) ? (1 << 30) : t2),
+                                           p->n_sms, st, &p->launches));
     } else {
       const int bn = gemm_tile_cols();
       const long long t1 = m_tiles_bound * ((g1.N + bn - 1) / bn), t2 = m_tiles_bound * ((g2.N + bn - 1) / bn);
@@ -296,10 +306,11 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     sl.lp.row_of_pair = reinterpret_cast<int32_t*>(b + L.row_of_pair);
     sl.lp.pair_of_row = reinterpret_cast<int32_t*>(b + L.pair_of_row);
     sl.lp.status = reinterpret_cast<int32_t*>(p->ws + L.status);
+    sl.lp.sched = reinterpret_cast<int32_t*>(b + L.sched);
     sl.xp = b + L.xp; sl.xp_scales = reinterpret_cast<float*>(b + L.xp_scales);
     sl.act = b + L.act; sl.act_scales = reinterpret_cast<float*>(b + L.act_scales);
     sl.y = b + L.y;
-    if (cfg->gemm_impl == CEP_GEMM_TCGEN05) {
+    if (cfg->gemm_impl != CEP_GEMM_SIMT) {
       int r1 = make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
       int r2 = make_operand_map(&sl.tm_a2, sl.act, elt, cfg->inter, L.cap_rows, 0, gemm_tile_rows());
       if (r1 || r2) {
@@ -335,10 +346,12 @@ int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const vo
   p->w2p = static_cast<uint8_t*>(packed) + P.w2;
   CUDA_TRY(p, launch_prepack(c, w_gate, w_up, w_down, p->w13p, p->w2p, st, &p->launches));
   CUDA_TRY(p, cudaEventRecord(p->weights_evt, st));
-  if (c.gemm_impl == CEP_GEMM_TCGEN05) {
+  if (c.gemm_impl != CEP_GEMM_SIMT) {
     const int elt = fp8 ? 1 : 2;
-    int r1 = make_operand_map(&p->tm_b1, p->w13p, elt, c.hidden, 2 * c.inter, c.n_experts_local, gemm_tile_cols());
-    int r2 = make_operand_map(&p->tm_b2, p->w2p, elt, c.inter, c.hidden, c.n_experts_local, gemm_tile_cols());
+    // the CTA-pair kernel loads half a weight tile per CTA
+    const int box = c.gemm_impl == CEP_GEMM_TCGEN05 ? gemm_tile_cols() / 2 : gemm_tile_cols();
+    int r1 = make_operand_map(&p->tm_b1, p->w13p, elt, c.hidden, 2 * c.inter, c.n_experts_local, box);
+    int r2 = make_operand_map(&p->tm_b2, p->w2p, elt, c.inter, c.hidden, c.n_experts_local, box);
     if (r1 || r2) return fail(p, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the weight operands failed (%d, %d)", r1, r2);
   }
   p->have_weights = true;
@@ -501,11 +514,11 @@ int moe_plan_destroy(cep_plan* p) {
   return CEP_OK;
 }
 
-int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n, int32_t tile,
-                          int32_t* expert, int32_t* m_block, int32_t* n_block) {
+int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n, int32_t n_group,
+                          int32_t tile, int32_t* expert, int32_t* m_block, int32_t* n_block) {
   if (!tile_prefix || n_experts <= 0 || !expert || !m_block || !n_block) return CEP_ERR_ARG;
   TileCoord tc;
-  if (!decode_tile(tile_prefix, n_experts, n_blocks_n, tile, &tc)) return CEP_ERR_ARG;
+  if (!decode_tile(tile_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) return CEP_ERR_ARG;
   *expert = tc.expert; *m_block = tc.m_block; *n_block = tc.n_block;
   return CEP_OK;
 }

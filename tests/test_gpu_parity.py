@@ -12,7 +12,7 @@ from helpers import (batch_ids, check_close, chunks_of, make_layer, run_layer, t
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [cep.CEP_GEMM_SIMT, cep.CEP_GEMM_TCGEN05]
+IMPLS = [cep.CEP_GEMM_SIMT, cep.CEP_GEMM_TCGEN05, cep.CEP_GEMM_TCGEN05_1CTA]
 
 
 def load(layer, inp):
@@ -30,7 +30,7 @@ def assert_layout_matches(layer, inv, ids_np, E):
 
 
 # ------------------------------------------------------------------ config 0 (tiny), whole tensor
-@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05", "tcgen05_1cta"])
 def test_tiny_sync_matches_oracle(impl):
     cfg = wl.CONFIGS["tiny"]
     host = wl.make_inputs(cfg)
@@ -45,7 +45,7 @@ def test_tiny_sync_matches_oracle(impl):
     layer.close()
 
 
-@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05", "tcgen05_1cta"])
 def test_tiny_chunked_equals_one_shot_bitwise_and_layouts_per_invocation(impl):
     cfg = wl.CONFIGS["tiny"]
     host = wl.make_inputs(cfg)
@@ -97,7 +97,7 @@ EDGE_CASES = {
 }
 
 
-@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("impl", IMPLS, ids=["simt", "tcgen05", "tcgen05_1cta"])
 @pytest.mark.parametrize("case", sorted(EDGE_CASES))
 def test_edge_cases(case, impl):
     host = EDGE_CASES[case]()
@@ -180,6 +180,8 @@ def test_simt_and_tensor_core_paths_agree_closely_on_mid():
         layer.close()
     rel = (outs[0] - outs[1]).norm() / outs[0].norm()
     assert rel < 3e-3            # both round the intermediate and the output to bf16 once
+    # the two tensor-core variants accumulate every row in the same K order: identical bits
+    assert torch.equal(outs[1], outs[2])
 
 
 # ------------------------------------------------------------------ errors are reported, never faults

@@ -27,13 +27,14 @@ def test_library_loads_and_exports_every_declared_symbol():
     assert sorted(names) == sorted(cep.binding.EXPORTS)
 
 
+@pytest.mark.parametrize("ng", [0, 1, 3, 8])
 @pytest.mark.parametrize("mt,nb", [([3, 0, 17, 1, 0, 40], 4), ([1], 1), ([0, 0, 5], 16), ([33, 16, 15], 3)])
-def test_tile_decode_covers_every_tile_exactly_once(mt, nb):
+def test_tile_decode_covers_every_tile_exactly_once(mt, nb, ng):
     prefix = np.concatenate([[0], np.cumsum(mt)]).astype(np.int32)
     total = int(prefix[-1]) * nb
     seen = set()
     for t in range(total):
-        e, m, n = cep.cep_debug_decode_tile(prefix, nb, t)
+        e, m, n = cep.cep_debug_decode_tile(prefix, nb, t, ng)
         assert 0 <= m < mt[e] and 0 <= n < nb
         seen.add((e, m, n))
     assert len(seen) == total
@@ -42,21 +43,23 @@ def test_tile_decode_covers_every_tile_exactly_once(mt, nb):
     # tiles of one expert are contiguous and experts appear in order
     last_e = -1
     for t in range(total):
-        e = cep.cep_debug_decode_tile(prefix, nb, t)[0]
+        e = cep.cep_debug_decode_tile(prefix, nb, t, ng)[0]
         assert e >= last_e
         last_e = e
 
 
-def test_tile_decode_group_order_shares_weight_tiles():
-    # inside a group of 16 m-tiles the n block is the slow index
-    prefix = np.array([0, 40], np.int32)
-    first = [cep.cep_debug_decode_tile(prefix, 4, t) for t in range(16)]
-    assert all(f[2] == 0 for f in first) and [f[1] for f in first] == list(range(16))
-    assert cep.cep_debug_decode_tile(prefix, 4, 16) == (0, 0, 1)
-    assert cep.cep_debug_decode_tile(prefix, 4, 64) == (0, 16, 0)
-    # the ragged last group (8 m-tiles) still enumerates all its tiles
-    assert cep.cep_debug_decode_tile(prefix, 4, 128) == (0, 32, 0)
-    assert cep.cep_debug_decode_tile(prefix, 4, 136) == (0, 32, 1)
+def test_tile_decode_order_keeps_an_experts_weight_panel_hot():
+    # inside an expert the n block is the fast index: consecutive tiles sweep all n blocks of one m block
+    prefix = np.array([0, 40, 43], np.int32)
+    assert [cep.cep_debug_decode_tile(prefix, 4, t) for t in range(5)] == \
+        [(0, 0, 0), (0, 0, 1), (0, 0, 2), (0, 0, 3), (0, 1, 0)]
+    assert cep.cep_debug_decode_tile(prefix, 4, 159) == (0, 39, 3)
+    assert cep.cep_debug_decode_tile(prefix, 4, 160) == (1, 0, 0)
+    assert cep.cep_debug_decode_tile(prefix, 4, 171) == (1, 2, 3)
+    # chunks of 3 n blocks: the chunk is swept over every m block before the next chunk starts
+    p2 = np.array([0, 2], np.int32)
+    assert [cep.cep_debug_decode_tile(p2, 4, t, 3) for t in range(8)] == \
+        [(0, 0, 0), (0, 0, 1), (0, 0, 2), (0, 1, 0), (0, 1, 1), (0, 1, 2), (0, 0, 3), (0, 1, 3)]
 
 
 @pytest.mark.parametrize("seed", range(6))
@@ -82,7 +85,7 @@ def test_config_validation_and_sizes():
     assert cep.moe_packed_weight_bytes(good) >= 8 * 3 * 512 * 256 * 2
     bad = [dict(hidden=500), dict(inter=100), dict(n_experts_local=9), dict(top_k=0), dict(top_k=33),
            dict(max_tokens=0), dict(mode=7), dict(n_streams=0), dict(threshold_pairs=-1), dict(dtype=5),
-           dict(gemm_impl=3), dict(n_experts_local=2000, n_experts_global=4000)]
+           dict(gemm_impl=4), dict(n_experts_local=2000, n_experts_global=4000)]
     for kw in bad:
         c = cep.CepConfig(512, 256, 8, 8, 2, 256, 2, 0, 0, 2, 0, 0, 0)
         for k_, v in kw.items():
