@@ -150,6 +150,43 @@ def run_reference(args):
     return 0
 
 
+def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
+    """Completion latency of Sync / Async / Async+streamFFN when the chunks arrive at seeded offsets
+    (lognormal, scaled to tau x the one-shot time), and the matched-work retention at tau = 0."""
+    import torch
+    from paper_2609_33252_b200.arrivals import run_with_arrivals
+    theta = args.theta if args.theta >= 0 else cfg.E_local * 1024
+    rstreams = [torch.cuda.Stream() for _ in chunks]
+    modes = [("sync", cep.CEP_MODE_SYNC, 0, 1), ("async", cep.CEP_MODE_ASYNC, 0, 1),
+             ("streamffn", cep.CEP_MODE_STREAMFFN, theta, args.streams)]
+    layers = {}
+    for name, mode, th, S in modes:
+        L = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, mode=mode,
+                         n_streams=S, threshold_pairs=th, gemm_impl=args.gemm_impl)
+        L.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+        layers[name] = L
+    torch.cuda.synchronize()
+    base = inp.arrival
+    report = {"theta_pairs": theta, "streams": args.streams, "t_sync_ms": t_sync_s * 1e3,
+              "arrival_offsets_unitless": base, "cases": []}
+    for tau in (0.0, 0.25, 0.5, 1.0):
+        arr = [tau * t_sync_s * a for a in base]
+        case = {"tau": tau, "last_arrival_ms": max(arr) * 1e3}
+        for name, _, _, _ in modes:
+            ts, ninv = [], 0
+            for rep in range(6):
+                dt, ninv = run_with_arrivals(layers[name], out, chunks, arr, ch_pairs, rstreams)
+                if rep >= 2:
+                    ts.append(dt)
+            case[name] = {"completion_ms": statistics.median(ts) * 1e3, "min_ms": min(ts) * 1e3, "invocations": ninv}
+        report["cases"].append(case)
+    c0 = report["cases"][0]
+    report["matched_work_retention"] = {m: c0["sync"]["completion_ms"] / c0[m]["completion_ms"] for m in ("async", "streamffn")}
+    for L in layers.values():
+        L.close()
+    return report
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -162,6 +199,8 @@ def main():
     ap.add_argument("--gemm-impl", type=int, default=0, help="0: CTA-pair tcgen05 (product), 2: one-CTA tcgen05")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-stream", action="store_true", help="skip the arrival-offset (streamFFN) section")
+    ap.add_argument("--theta", type=int, default=-1, help="streamFFN threshold in local pairs (default: E_local*1024)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3 if args.impl == "ours" else args.warmup
@@ -291,6 +330,11 @@ def main():
         e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": hout.numel() * 2}
 
+    # ---- chunked asynchronous execution under seeded arrival offsets (rank 0 only, outside the timed step)
+    stream_report = None
+    if rank == 0 and not args.no_stream and cfg.n_chunks > 1:
+        stream_report = stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, ms * 1e-3, args)
+
     if rank != 0:
         layer.close()
         if dist is not None:
@@ -337,7 +381,7 @@ def main():
                              (3.0 * cfg.H * cfg.I * 2 * cfg.E_local / 1e9)},
             "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal_2250": ffn_tflops / NOMINAL_BF16_TFLOPS,
                            "frac_of_measured": ffn_tflops / peak_tf, "flops_per_step": work["flops"]},
-            "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e,
+            "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e, "streamffn": stream_report,
             "gpu_launches": int(launches)}
     if not args.no_cpu_baseline:
         import oracle
