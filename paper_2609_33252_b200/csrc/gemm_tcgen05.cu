@@ -186,7 +186,10 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       TileCoord tc;
       if (!decode_tile(tile_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-      if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status)) break;
+      // the lanes may leave the polling loop in different iterations; the tensor-memory loads below are
+      // warp-collective (.sync.aligned), so the warp must be converged again before it issues them
+      const bool got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
+      if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
                              tc.m_block * BM + lane_grp * 32 + lane, tc.expert, tc.n_block, n_out_cols, out_ld, out,
@@ -228,6 +231,7 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
 constexpr int kPairStages = CEP_PAIR_STAGES;
 constexpr int PB_STAGE = (BN / 2) * BKB;               // 16 KiB: this CTA's half of the weight tile
 constexpr int kMaxExperts = 1024;
+constexpr int kTilePoison = -2;
 constexpr int kSchedRing = 4;                          // tile ids in flight between the scheduler and its readers
 constexpr int kSchedReaders = 11;                      // leader: producer, MMA, 4 epilogue warps; peer: producer, 4 epilogue warps
 constexpr int kPairThreads = 224;                      // warp 6 of the leader CTA hands out tiles
@@ -249,7 +253,14 @@ struct TileReader {
     const uint32_t bar = smem_u32(&bars->sched_full[slot]);
     const bool ok = is_peer ? mbar_wait_acq_cluster(bar, phase, abort_flag, status) : mbar_wait(bar, phase, abort_flag, status);
     if (!ok) return -1;
-    return bars->sched_tile[slot];
+    const int t = bars->sched_tile[slot];
+    if (t < -1) {                              // a slot read before its value arrived: report, never use it
+      atomicExch(&status[kStDetail], 0x5C4ED);
+      atomicExch(&status[kStTimeout], 1);
+      *abort_flag = 1;
+      return -1;
+    }
+    return t;
   }
   // Frees the ring slot for the scheduler (one arrival per reading role) and advances.
   __device__ __forceinline__ void done(PairBarriers* bars, bool signal) {
@@ -280,7 +291,12 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPairStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), 8); }
-    for (int s = 0; s < kSchedRing; ++s) { mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders); }
+    for (int s = 0; s < kSchedRing; ++s) {
+      mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders);
+#ifndef CEP_EXP_NO_POISON
+      bars->sched_tile[s] = kTilePoison;     // shared memory keeps what the previous CTA on this SM left
+#endif
+    }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -413,7 +429,10 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
       if (tile < 0) break;
       TileCoord tc;
       if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-      if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status)) break;
+      // the lanes may leave the polling loop in different iterations; the tensor-memory loads below are
+      // warp-collective (.sync.aligned), so the warp must be converged again before it issues them
+      const bool got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
+      if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
                              tc.m_block * (2 * BM) + (int)rank * BM + lane_grp * 32 + lane, tc.expert, tc.n_block,
