@@ -89,7 +89,7 @@ class ClockSampler:
 def workload_numbers(cfg, n_pairs):
     """Algorithmic work of one step ('Algorithmic work per unit')."""
     H, I, T, E = cfg.H, cfg.I, cfg.T, cfg.E_local
-    s = 2
+    s = 2 if cfg.dtype == "bf16" else 1 + 4.0 / 128      # bytes per element (fp8: code + its share of a 1x128 scale)
     return {
         "pairs": n_pairs,
         "flops": 6.0 * H * I * n_pairs,
@@ -162,6 +162,7 @@ def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
     layers = {}
     for name, mode, th, S in modes:
         L = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, mode=mode,
+                         dtype=cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16,
                          n_streams=S, threshold_pairs=th, gemm_impl=args.gemm_impl)
         L.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
         layers[name] = L
@@ -234,7 +235,8 @@ def main():
     work = workload_numbers(cfg, n_pairs)
     ch_pairs = [int((inp.topk_ids[o:o + n] < cfg.E_local).sum().item()) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
 
-    layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks,
+    dt = cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16
+    layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
                          mode=cep.CEP_MODE_SYNC, n_streams=args.streams, profile_kernels=1,
                          gemm_impl=args.gemm_impl)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
@@ -296,6 +298,8 @@ def main():
         hx = inp.x.cpu().pin_memory(); hid = inp.topk_ids.cpu().pin_memory(); hw = inp.topk_w.cpu().pin_memory()
         hout = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory()
         dx, did, dw = torch.empty_like(inp.x), torch.empty_like(inp.topk_ids), torch.empty_like(inp.topk_w)
+        hxs = None if inp.x_scale is None else inp.x_scale.cpu().pin_memory()
+        dxs = None if inp.x_scale is None else torch.empty_like(inp.x_scale)
         rstreams = [torch.cuda.Stream() for _ in chunks]
         main = torch.cuda.current_stream()
 
@@ -308,7 +312,10 @@ def main():
                     dx[o:o + n].copy_(hx[o:o + n], non_blocking=True)
                     did[o:o + n].copy_(hid[o:o + n], non_blocking=True)
                     dw[o:o + n].copy_(hw[o:o + n], non_blocking=True)
-                cep.ffn_submit_chunk(layer.plan, c, o, n, dx[o:o + n], None, did[o:o + n], dw[o:o + n], ch_pairs[c], st)
+                    if dxs is not None:
+                        dxs[o:o + n].copy_(hxs[o:o + n], non_blocking=True)
+                cep.ffn_submit_chunk(layer.plan, c, o, n, dx[o:o + n], None if dxs is None else dxs[o:o + n],
+                                     did[o:o + n], dw[o:o + n], ch_pairs[c], st)
             cep.ffn_flush(layer.plan)
             cep.combine(layer.plan, main)
             hout.copy_(out, non_blocking=True)
@@ -326,7 +333,7 @@ def main():
             t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e_ms = float(t.item())
-        h2d = hx.numel() * 2 + hid.numel() * 4 + hw.numel() * 4
+        h2d = hx.numel() * hx.element_size() + hid.numel() * 4 + hw.numel() * 4 + (0 if hxs is None else hxs.numel() * 4)
         e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": hout.numel() * 2}
 
@@ -351,10 +358,15 @@ def main():
     sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
     sustained = (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
     peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-    roofline = {"bound": "tensor", "kernel": "grouped_gemm_bf16_kernel<swiglu> (GEMM1: gate/up + SiLU*up)",
+    nominal_tf = NOMINAL_BF16_TFLOPS
+    if cfg.dtype == "fp8":          # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2)
+        peak_tf, nominal_tf = 2.0 * peak_tf, 2.0 * NOMINAL_BF16_TFLOPS
+    roofline = {"bound": "tensor", "kernel": "grouped GEMM1 (gate/up + SiLU*up%s), CTA-pair tcgen05" %
+                          (" + e4m3 re-quantisation" if cfg.dtype == "fp8" else ""),
                 "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
-                "peak_kind": ("sustained" if sustained else "burst") + " bf16 cuBLAS, of " + peaks["source"],
-                "frac_of_nominal_2250": g1_tflops / NOMINAL_BF16_TFLOPS,
+                "peak_kind": ("sustained" if sustained else "burst") + " bf16 cuBLAS" +
+                             (" x2 (nominal fp8:bf16 ratio)" if cfg.dtype == "fp8" else "") + ", of " + peaks["source"],
+                "frac_of_nominal": g1_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                 "duration_ms": g1_ms, "traffic": None}
     prof = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(prof):
@@ -378,8 +390,8 @@ def main():
                        "E_global": cfg.E_global, "top_k": cfg.k, "local_pairs": n_pairs, "chunks": list(cfg.chunks),
                        "mode": "sync (one invocation, all chunks present)", "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (weights %.2f GB re-read every step)" %
-                             (3.0 * cfg.H * cfg.I * 2 * cfg.E_local / 1e9)},
-            "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal_2250": ffn_tflops / NOMINAL_BF16_TFLOPS,
+                             (3.0 * cfg.H * cfg.I * (2 if cfg.dtype == "bf16" else 1) * cfg.E_local / 1e9)},
+            "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal": ffn_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                            "frac_of_measured": ffn_tflops / peak_tf, "flops_per_step": work["flops"]},
             "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e, "streamffn": stream_report,
             "gpu_launches": int(launches)}

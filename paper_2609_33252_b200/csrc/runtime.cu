@@ -138,6 +138,7 @@ struct cep_plan {
   cudaEvent_t begin_evt, readback_evt, weights_evt;
   bool have_weights, layer_open, flushed, readback_pending, ever_closed;
   uint8_t* w13p; uint8_t* w2p;
+  float* s13p; float* s2p;                      // fp8: packed weight scales
   GemmTensorMap tm_b1, tm_b2;
   // current layer call
   void* out; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
@@ -199,6 +200,15 @@ int launch_invocation(cep_plan* p) {
       CUDA_TRY(p, launch_gemm_simt(g1, sl.xp, p->w13p, sl.act, sl.lp, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
       CUDA_TRY(p, launch_gemm_simt(g2, sl.act, p->w2p, sl.y, sl.lp, st, &p->launches));
+    } else if (c.gemm_impl == CEP_GEMM_TCGEN05 && fp8) {
+      const int bn = gemm_tile_cols();
+      const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
+      const long long t1 = pair_bound * ((g1.N + bn - 1) / bn), t2 = pair_bound * ((g2.N + bn - 1) / bn);
+      CUDA_TRY(p, launch_gemm_fp8_pair(g1, sl.tm_a1, p->tm_b1, sl.xp_scales, p->s13p, sl.act, sl.act_scales, sl.lp,
+                                       (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
+      if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
+      CUDA_TRY(p, launch_gemm_fp8_pair(g2, sl.tm_a2, p->tm_b2, sl.act_scales, p->s2p, sl.y, nullptr, sl.lp,
+                                       (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
     } else if (c.gemm_impl == CEP_GEMM_TCGEN05) {
       const int bn = gemm_tile_cols();
       const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
@@ -258,8 +268,11 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   if (!out) return fail(nullptr, CEP_ERR_ARG, "out is NULL");
   *out = nullptr;
   if (!workspace) return fail(nullptr, CEP_ERR_ARG, "workspace is NULL");
-  if (cfg->dtype == CEP_FP8_E4M3_BLOCK128)
-    return fail(nullptr, CEP_ERR_UNSUPPORTED, "the block-scaled fp8 path is not built yet");
+  if (cfg->dtype == CEP_FP8_E4M3_BLOCK128) {
+    if (cfg->gemm_impl != CEP_GEMM_TCGEN05)
+      return fail(nullptr, CEP_ERR_UNSUPPORTED, "block-scaled fp8 runs on the CTA-pair tensor-core kernel only");
+    if (cfg->hidden % 256) return fail(nullptr, CEP_ERR_ARG, "fp8 needs hidden to be a multiple of 256");
+  }
   Layout L = make_layout(*cfg);
   if (workspace_bytes < L.total) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace must be 256-byte aligned");
@@ -344,7 +357,10 @@ int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const vo
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   p->w13p = static_cast<uint8_t*>(packed) + P.w13;
   p->w2p = static_cast<uint8_t*>(packed) + P.w2;
+  p->s13p = reinterpret_cast<float*>(static_cast<uint8_t*>(packed) + P.s13);
+  p->s2p = reinterpret_cast<float*>(static_cast<uint8_t*>(packed) + P.s2);
   CUDA_TRY(p, launch_prepack(c, w_gate, w_up, w_down, p->w13p, p->w2p, st, &p->launches));
+  if (fp8) CUDA_TRY(p, launch_pack_scales(c, s_gate, s_up, s_down, p->s13p, p->s2p, st, &p->launches));
   CUDA_TRY(p, cudaEventRecord(p->weights_evt, st));
   if (c.gemm_impl != CEP_GEMM_SIMT) {
     const int elt = fp8 ? 1 : 2;
