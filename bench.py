@@ -102,6 +102,16 @@ def workload_numbers(cfg, n_pairs):
     }
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Every rank contributes its own time; the job's time is the slowest rank's."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def host_copy(inp):
     """The same inputs with every tensor on the host (for the CPU oracle)."""
     import dataclasses
@@ -285,11 +295,7 @@ def main():
             for k_ in kern:
                 kern[k_].append(getattr(info, k_))
     clocks = sampler.stop() if rank == 0 else None
-    ms = total_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(total_ms / args.steps, dist, "cuda")
     value = world * cfg.T / (ms * 1e-3)
 
     # ---- end to end: pinned host buffers -> device -> path -> host, every step
@@ -328,11 +334,7 @@ def main():
             e2e_step()
         ev1.record()
         barrier()
-        e2e_ms = ev0.elapsed_time(ev1) / args.steps
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / args.steps, dist, "cuda")
         h2d = hx.numel() * hx.element_size() + hid.numel() * 4 + hw.numel() * 4 + (0 if hxs is None else hxs.numel() * 4)
         e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": hout.numel() * 2}

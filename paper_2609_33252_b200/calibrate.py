@@ -1,0 +1,81 @@
+"""Launch-threshold calibration (Section 3.2 "Launch threshold"; Section 4.2 FFN latency model).
+
+Profiles the expert-FFN throughput of THIS library on THIS GPU as a function of the expert-token
+count of one invocation (uniform rows per expert, the shapes of a configuration), and sets theta to the
+smallest profiled count that reaches a fraction rho of the observed peak.  Also returns the normalised
+efficiency eta(N) = throughput(N) / peak, from which the paper's FFN latency model
+F(N) = N / (eta(N) * P_peak) follows.  This is a measurement harness over the C ABI: every timed
+kernel is the library's.
+"""
+from __future__ import annotations
+
+import json
+import statistics
+import sys
+from typing import Dict, List, Sequence
+
+from . import binding as cep
+from . import workloads as wl
+
+
+def uniform_routing(rows_per_expert: int, E: int, k: int, device):
+    """ids [T,k] giving every local expert exactly rows_per_expert rows (T = rows*E/k tokens)."""
+    import torch
+    T = max(1, rows_per_expert * E // k)
+    t = torch.arange(T, device=device, dtype=torch.int64)[:, None]
+    j = torch.arange(k, device=device, dtype=torch.int64)[None, :]
+    ids = ((t * k + j) % E).to(torch.int32).contiguous()
+    w = torch.full((T, k), 1.0 / k, dtype=torch.float32, device=device)
+    return ids, w
+
+
+def profile(cfg: wl.MoEConfig, rows: Sequence[int] = (16, 32, 64, 128, 256, 512, 1024, 2048, 4096),
+            reps: int = 5, device="cuda") -> List[Dict]:
+    import torch
+    inp = wl.make_inputs(wl.scaled(cfg, T=8, chunks=(8,)), device=device, keep_logits=False)   # weights only
+    E, k, H, I = cfg.E_local, min(cfg.k, cfg.E_local), cfg.H, cfg.I
+    fp8 = cfg.dtype == "fp8"
+    max_T = max(rows) * E // k
+    layer = cep.MoELayer(H, I, E, E, k, max_T, 1, dtype=cep.CEP_FP8_E4M3_BLOCK128 if fp8 else cep.CEP_BF16,
+                         mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+    g = torch.Generator(device=device).manual_seed(wl.SEED_BASE + 99)
+    out_rows = []
+    for m in rows:
+        ids, w = uniform_routing(m, E, k, device)
+        T = ids.shape[0]
+        x32 = torch.randn((T, H), generator=g, device=device)
+        if fp8:
+            x, xs = wl.quantize_rows_1x128(x32)
+        else:
+            x, xs = x32.to(torch.bfloat16), None
+        out = torch.empty((T, H), dtype=torch.bfloat16, device=device)
+        g1, g2, tot = [], [], []
+        for r in range(reps + 2):
+            layer.run(out, [(0, x, xs, ids, w)])
+            torch.cuda.synchronize()
+            info = cep.ffn_query(layer.plan, 0)
+            if r >= 2:
+                g1.append(info.gemm1_ms); g2.append(info.gemm2_ms); tot.append(info.elapsed_ms)
+        pairs = T * k
+        ffn_ms = statistics.median(g1) + statistics.median(g2)
+        out_rows.append({"rows_per_expert": m, "expert_tokens": pairs, "ffn_ms": ffn_ms,
+                         "layer_ms": statistics.median(tot), "tflops": 6.0 * H * I * pairs / (ffn_ms * 1e-3) / 1e12})
+    layer.close()
+    return out_rows
+
+
+def calibrate(cfg: wl.MoEConfig, rho: float = 0.90, **kw) -> Dict:
+    """theta = smallest profiled expert-token count whose throughput is >= rho * observed peak."""
+    prof = profile(cfg, **kw)
+    peak = max(p["tflops"] for p in prof)
+    for p in prof:
+        p["eta"] = p["tflops"] / peak
+    theta = next(p["expert_tokens"] for p in prof if p["eta"] >= rho)
+    return {"config": cfg.name, "rho": rho, "peak_tflops": peak, "theta_pairs": theta,
+            "theta_rows_per_expert": theta // cfg.E_local, "profile": prof}
+
+
+if __name__ == "__main__":
+    name = sys.argv[1] if len(sys.argv) > 1 else "ep_shard"
+    print(json.dumps(calibrate(wl.CONFIGS[name])))

@@ -243,18 +243,25 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
         if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
         tc_fence_after();
         const uint32_t t_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN);
+        // two 32-column loads in flight per wait; the scratch buffer is handed back to the MMA warp as
+        // soon as its last column has been read, before the final multiply-adds
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t v[32];
-          tc_ld32(t_addr + (uint32_t)((c < 2 ? col0 : col1) + (c & 1) * 32), v);
+        for (int g = 0; g < 2; ++g) {
+          uint32_t v0[32], v1[32];
+          tc_ld32(t_addr + (uint32_t)(g == 0 ? col0 : col1), v0);
+          tc_ld32(t_addr + (uint32_t)((g == 0 ? col0 : col1) + 32), v1);
           tc_wait_ld();
-          const float s = c < 2 ? s0 : s1;
+          if (g == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
+          }
+          const float s = g == 0 ? s0 : s1;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(__uint_as_float(v[i]), s, acc[c * 32 + i]);
+          for (int i = 0; i < 32; ++i) acc[g * 64 + i] = fmaf(__uint_as_float(v0[i]), s, acc[g * 64 + i]);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[g * 64 + 32 + i] = fmaf(__uint_as_float(v1[i]), s, acc[g * 64 + 32 + i]);
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
         if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
       }
       if (!ok) break;

@@ -74,6 +74,8 @@ CONFIGS = {
     # enough for multi-pass profiler captures while its weights (0.7 GB) still exceed the L2
     "ep_shard_small": MoEConfig("ep_shard_small", 2, T=2048, H=7168, I=2048, E_global=64, E_local=8, k=8,
                                 chunks=tuple(_equal_chunks(2048, 8)), zipf_s=1.1),
+    "fp8_shard_small": MoEConfig("fp8_shard_small", 4, T=2048, H=7168, I=3072, E_global=64, E_local=8, k=8,
+                                 chunks=tuple(_equal_chunks(2048, 8)), dtype="fp8", zipf_s=1.1),
     "fp8_shard": MoEConfig("fp8_shard", 4, T=32768, H=7168, I=3072, E_global=512, E_local=64, k=8,
                            chunks=tuple(_equal_chunks(32768, 8)), dtype="fp8", zipf_s=1.1),
 }
