@@ -26,6 +26,10 @@ if ROOT not in sys.path:
 METRIC = "MoE-layer prefill tokens/s (streamFFN routed-expert path: permute + grouped SwiGLU expert FFN + combine)"
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one GEMM1 launch, from the ncu captures summarised in
+# profiles/grouped_gemm_bf16_pair_ep_shard.md and profiles/grouped_gemm_fp8_pair_fp8_shard_small.md
+GEMM1_DRAM_TRAFFIC = {"ep_shard": 5.64e9 + 0.51e9, "straggler": 5.64e9 + 0.51e9,
+                      "ep_shard_small": 1.02e9 + 0.041e9, "fp8_shard_small": 0.462e9 + 0.034e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -370,13 +374,7 @@ def main():
                              (" x2 (nominal fp8:bf16 ratio)" if cfg.dtype == "fp8" else "") + ", of " + peaks["source"],
                 "frac_of_nominal": g1_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                 "duration_ms": g1_ms, "traffic": None}
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(prof):
-        try:
-            tr = json.load(open(prof)).get(cfg.name, {})
-            roofline["traffic"] = tr.get("gemm1_dram_bytes_per_launch")
-        except Exception:
-            pass
+    roofline["traffic"] = GEMM1_DRAM_TRAFFIC.get(cfg.name)
     kernels = {
         "layout": {"ms": med["layout_ms"], "GB/s": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9,
                    "frac_of_hbm": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
