@@ -188,7 +188,7 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
       if (!decode_tile(tile_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
       // the lanes may leave the polling loop in different iterations; the tensor-memory loads below are
       // warp-collective (.sync.aligned), so the warp must be converged again before it issues them
-      const bool got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
+      const bool got = mbar_wait_relaxed(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
       if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
@@ -201,9 +201,6 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
     }
   }
   // ------------------------------------------------------------------ teardown
-#ifdef CEP_EXP_TIMESTAMPS
-  if (threadIdx.x == 64) status[8 + blockIdx.x] = (int32_t)(globaltimer() >> 8);     // 256 ns units
-#endif
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -251,7 +248,7 @@ struct TileReader {
   // Waits for the next tile id.  The caller must call done() once every thread of the role has the value.
   __device__ __forceinline__ int next(PairBarriers* bars, bool is_peer, volatile int* abort_flag, int32_t* status) {
     const uint32_t bar = smem_u32(&bars->sched_full[slot]);
-    const bool ok = is_peer ? mbar_wait_acq_cluster(bar, phase, abort_flag, status) : mbar_wait(bar, phase, abort_flag, status);
+    const bool ok = is_peer ? mbar_wait_acq_cluster(bar, phase, abort_flag, status) : mbar_wait_relaxed(bar, phase, abort_flag, status);
     if (!ok) return -1;
     const int t = bars->sched_tile[slot];
     if (t < -1) {                              // a slot read before its value arrived: report, never use it
@@ -293,9 +290,7 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), 8); }
     for (int s = 0; s < kSchedRing; ++s) {
       mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders);
-#ifndef CEP_EXP_NO_POISON
       bars->sched_tile[s] = kTilePoison;     // shared memory keeps what the previous CTA on this SM left
-#endif
     }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -337,9 +332,6 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
         const int row0 = padded_offsets[tc.expert] + tc.m_block * (2 * BM) + (int)rank * BM;
         const int n0 = tc.n_block * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
-#ifdef CEP_EXP_NO_LOAD
-          ok = false; break;
-#endif
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
           const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);        // the leader's barrier
           // the leader alone arrives, announcing both CTAs' bytes; the peer's bytes can only land in
@@ -367,34 +359,18 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-#ifndef CEP_EXP_NO_LOAD
           if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status)) { ok = false; break; }
-#endif
           tc_fence_after();
           const uint64_t adesc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE));
           const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * PB_STAGE));
-#ifndef CEP_EXP_NO_MMA
 #pragma unroll
           for (int k4 = 0; k4 < BKB / 32; ++k4)
             tc_mma_f16_pair(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, (kb | k4) != 0 ? 1u : 0u);
-#endif
-#ifdef CEP_PAIR_TWO_COMMITS
-          const uint32_t e_bar = smem_u32(&bars->empty[stage]);
-          tc_commit_pair(mapa(e_bar, 0));               // frees the stage in both CTAs
-          tc_commit_pair(mapa(e_bar, 1));
-#else
           tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);   // frees the stage in both CTAs
-#endif
           if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-#ifdef CEP_PAIR_TWO_COMMITS
-        const uint32_t f_bar = smem_u32(&bars->acc_full[acc]);
-        tc_commit_pair(mapa(f_bar, 0));                 // accumulator complete, both halves
-        tc_commit_pair(mapa(f_bar, 1));
-#else
         tc_commit_pair_both(smem_u32(&bars->acc_full[acc]), 3);  // accumulator complete, both halves
-#endif
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -406,7 +382,7 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
     if (lane == 0 && !is_peer) {
       int slot = 0; uint32_t phase = 0;
       for (;;) {
-        if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1u, abort_flag, status)) break;
+        if (!mbar_wait_relaxed(smem_u32(&bars->sched_empty[slot]), phase ^ 1u, abort_flag, status)) break;
         int t = atomicAdd(tile_counter, 1);
         if (t >= total_tiles) t = -1;
         bars->sched_tile[slot] = t;
@@ -431,7 +407,7 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
       if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
       // the lanes may leave the polling loop in different iterations; the tensor-memory loads below are
       // warp-collective (.sync.aligned), so the warp must be converged again before it issues them
-      const bool got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
+      const bool got = mbar_wait_relaxed(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, status);
       if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       epilogue_tile<kSwiglu>(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc * BN),
@@ -444,9 +420,6 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
     }
   }
   // ------------------------------------------------------------------ teardown
-#ifdef CEP_EXP_TIMESTAMPS
-  if (threadIdx.x == 64) status[8 + blockIdx.x] = (int32_t)(globaltimer() >> 8);     // 256 ns units
-#endif
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();               // no CTA leaves while its peer may still signal or read it

@@ -80,6 +80,17 @@ __host__ __device__ constexpr uint32_t make_idesc_e4m3(int m, int n) {
 __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory"); }
 __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory"); }
 
+// packed pairs of fp32: one instruction does two independent round-to-nearest multiply-adds
+__device__ __forceinline__ unsigned long long pack_f32x2(uint32_t lo, uint32_t hi) {
+  unsigned long long r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi)); return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long v, unsigned long long s) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(v), "l"(s));
+}
+
 // two e4m3 codes (round-to-nearest-even, saturating to +-448) from two floats: lo in bits 0-7
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
   uint16_t r;
@@ -218,7 +229,7 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
     int pb = 0; uint32_t pb_phase = 0;
     uint32_t tile_parity = 0;
     Ring rd;
-    float acc[128];
+    unsigned long long acc2[64];                       // 128 fp32 accumulators as packed pairs
     for (;;) {
       const int tile = rd.next(bars, is_peer, abort_flag, status);
       __syncwarp();
@@ -234,7 +245,7 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
       const float* sw0_p = b_scales + ((size_t)tc.expert * (2 * n_blocks_n) + nb0) * num_kb;
       const float* sw1_p = b_scales + ((size_t)tc.expert * (2 * n_blocks_n) + nb1) * num_kb;
 #pragma unroll
-      for (int i = 0; i < 128; ++i) acc[i] = 0.f;
+      for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
         const float sa = row_ok ? __ldg(sa_row + kb) : 0.f;
@@ -257,15 +268,19 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
             if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
           }
           const float s = g == 0 ? s0 : s1;
+          const unsigned long long s2 = pack_f32x2(__float_as_uint(s), __float_as_uint(s));
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc[g * 64 + i] = fmaf(__uint_as_float(v0[i]), s, acc[g * 64 + i]);
+          for (int i = 0; i < 16; ++i) fma_f32x2(acc2[g * 32 + i], pack_f32x2(v0[2 * i], v0[2 * i + 1]), s2);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc[g * 64 + 32 + i] = fmaf(__uint_as_float(v1[i]), s, acc[g * 64 + 32 + i]);
+          for (int i = 0; i < 16; ++i) fma_f32x2(acc2[g * 32 + 16 + i], pack_f32x2(v1[2 * i], v1[2 * i + 1]), s2);
         }
         if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
       }
       if (!ok) break;
       // ---------------------------------------------------------------- epilogue from registers
+      float acc[128];
+#pragma unroll
+      for (int i = 0; i < 64; ++i) unpack_f32x2(acc2[i], acc[2 * i], acc[2 * i + 1]);
       if (kSwiglu) {
         // acc[0..63] = gate cols, acc[64..127] = up cols -> 64 activations of this row
         float amax = 0.f;

@@ -47,6 +47,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// The same bounded wait for roles that wait long (a whole tile) and are not on the k-step critical path:
+// sleeps between polls so the waiting warps leave issue slots and power to the tensor pipe.
+#ifndef CEP_WAIT_SLEEP_NS
+#define CEP_WAIT_SLEEP_NS 0
+#endif
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t spin = 1;; ++spin) {
+    if (CEP_WAIT_SLEEP_NS > 0) __nanosleep(CEP_WAIT_SLEEP_NS);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 1023u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(&status[kStTimeout], 1);
+        return false;
+      }
+    }
+  }
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
