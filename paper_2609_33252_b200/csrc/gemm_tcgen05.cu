@@ -227,7 +227,10 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
 #endif
 constexpr int kPairStages = CEP_PAIR_STAGES;
 constexpr int PB_STAGE = (BN / 2) * BKB;               // 16 KiB: this CTA's half of the weight tile
-constexpr int kMaxExperts = 1024;
+#ifndef CEP_PAIR_MAXE
+#define CEP_PAIR_MAXE 1024
+#endif
+constexpr int kMaxExperts = CEP_PAIR_MAXE;
 constexpr int kTilePoison = -2;
 constexpr int kSchedRing = 4;                          // tile ids in flight between the scheduler and its readers
 constexpr int kSchedReaders = 11;                      // leader: producer, MMA, 4 epilogue warps; peer: producer, 4 epilogue warps

@@ -26,11 +26,12 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& 
                                      int64_t* launches);
 int gemm_pair_clusters();
 
-// Block-scaled e4m3 variant (CTA pairs).  a_scales [rows, K/128], b_scales [E, N/128, K/128] fp32.  With
-// p.swiglu the output is e4m3 codes [rows, N/2] plus out_scales [rows, N/256]; otherwise bf16 [rows, N].
-cudaError_t launch_gemm_fp8_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                                 const float* a_scales, const float* b_scales, void* out, float* out_scales,
-                                 const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s, int64_t* launches);
+// Block-scaled e4m3 variant.  a_scales [rows, K/128], b_scales [E, N/128, K/128] fp32.  With p.swiglu the output is
+// e4m3 codes [rows, N/2] plus out_scales [rows, N/256]; otherwise bf16 [rows, N].  pair != 0: CTA pairs on 256x256
+// tiles (weight map with a 128-row box); pair == 0: one CTA per 128x256 tile (256-row box).
+cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                            const float* a_scales, const float* b_scales, void* out, float* out_scales,
+                            const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches);
 // s13p[e][2*ib + (0 gate | 1 up)][kb] and s2p[e][hb][kb] from the caller's [E, in/128, out/128] scale tensors
 cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const float* s_up, const float* s_down,
                                float* s13p, float* s2p, cudaStream_t s, int64_t* launches);

@@ -29,20 +29,27 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128, BN = 256, BKB = 128;          // BKB bytes = 128 e4m3 elements = one scale block
-constexpr int kStages = 6;
 constexpr int A_STAGE = BM * BKB;                      // 16 KiB
-constexpr int PB_STAGE = (BN / 2) * BKB;               // 16 KiB: this CTA's half of the weight tile
+// kPair: CTA pairs (256x256 tiles, each CTA loads half of the weight tile, 6 stages of 32 KiB);
+// !kPair: one CTA per 128x256 tile (whole weight tile per CTA, 4 stages of 48 KiB): every hand-off
+// between the MMA warp and the promotion warps stays inside the SM
+template <bool kPair> struct Geo {
+  static constexpr int kStages = kPair ? 6 : 4;
+  static constexpr int B_STAGE = (kPair ? BN / 2 : BN) * BKB;
+  static constexpr int kRingReaders = kPair ? 19 : 10;    // producer, MMA, 8 promotion warps (+ peer: producer, 8)
+  static constexpr int kPartArrivals = kPair ? 16 : 8;
+  static constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE) + 256 + (1024 + 1) * 4 + 2 * 2 * BM * 4 + 1024;
+};
+constexpr int kMaxStages = 6;
 constexpr int kThreads = 384;
 constexpr int kPromoWarp0 = 4, kPromoWarps = 8;
 constexpr int kTmemCols = 512;
 constexpr int kMaxExperts = 1024;
 constexpr int kRing = 4;
 constexpr int kTilePoison = -2;
-// tile-ring readers: leader producer, MMA, 8 promotion warps; peer producer, 8 promotion warps
-constexpr int kRingReaders = 19;
 
 struct __align__(8) Bars {
-  uint64_t full[kStages], empty[kStages];
+  uint64_t full[kMaxStages], empty[kMaxStages];
   uint64_t part_full[2], part_empty[2];               // scratch accumulators in tensor memory
   uint64_t sched_full[kRing], sched_empty[kRing];
   uint64_t amax_bar[4];                               // per lane group: the two warps sharing its rows
@@ -51,7 +58,6 @@ struct __align__(8) Bars {
   int abort_flag;
 };
 static_assert(sizeof(Bars) <= 256, "barrier block");
-constexpr int kSmemBytes = kStages * (A_STAGE + PB_STAGE) + 256 + (kMaxExperts + 1) * 4 + 2 * 2 * BM * 4 + 1024;
 
 struct Ring {
   int slot = 0; uint32_t phase = 0;
@@ -63,14 +69,22 @@ struct Ring {
     if (t < -1) { atomicExch(&status[kStDetail], 0x5C4ED); atomicExch(&status[kStTimeout], 1); *abort_flag = 1; return -1; }
     return t;
   }
+  template <bool kPair>
   __device__ __forceinline__ void done(Bars* b, bool signal) {
-    if (signal) mbar_arrive_cluster(mapa(smem_u32(&b->sched_empty[slot]), 0));
+    if (signal) {
+      if (kPair) mbar_arrive_cluster(mapa(smem_u32(&b->sched_empty[slot]), 0));
+      else mbar_arrive(smem_u32(&b->sched_empty[slot]));
+    }
     if (++slot == kRing) { slot = 0; phase ^= 1u; }
   }
 };
 
 __device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
                ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // kind::f8f6f4: fp32 accumulate, e4m3 x e4m3 (format code 0), both operands K-major
@@ -98,9 +112,9 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
   return r;
 }
 
-template <bool kSwiglu>
+template <bool kSwiglu, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
-grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                              int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
                              const float* __restrict__ a_scales /*[rows, num_kb]*/,
                              const float* __restrict__ b_scales /*[E, N/128, num_kb]*/,
@@ -111,21 +125,23 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
                              int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int kStages = Geo<kPair>::kStages, B_STAGE = Geo<kPair>::B_STAGE;
+  constexpr int kRowsPerTile = kPair ? 2 * BM : BM;
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + kStages * A_STAGE;
-  Bars* bars = reinterpret_cast<Bars*>(smem + kStages * (A_STAGE + PB_STAGE));
-  int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kStages * (A_STAGE + PB_STAGE) + 256);
+  Bars* bars = reinterpret_cast<Bars*>(smem + kStages * (A_STAGE + B_STAGE));
+  int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kStages * (A_STAGE + B_STAGE) + 256);
   float* s_amax = reinterpret_cast<float*>(pair_prefix + kMaxExperts + 1);           // [tile parity][half][128]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;
   const bool is_peer = rank != 0;
   volatile int* abort_flag = &bars->abort_flag;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->part_full[s]), 1); mbar_init(smem_u32(&bars->part_empty[s]), 2 * kPromoWarps); }
+    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->part_full[s]), 1); mbar_init(smem_u32(&bars->part_empty[s]), Geo<kPair>::kPartArrivals); }
     for (int s = 0; s < kRing; ++s) {
-      mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kRingReaders);
+      mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), Geo<kPair>::kRingReaders);
       bars->sched_tile[s] = kTilePoison;
     }
     for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars->amax_bar[s]), 2);
@@ -134,18 +150,28 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
   }
   if (threadIdx.x == 32) {
     int run = 0;
-    for (int e = 0; e < n_experts; ++e) { pair_prefix[e] = run; run += (tile_prefix[e + 1] - tile_prefix[e] + 1) >> 1; }
+    for (int e = 0; e < n_experts; ++e) {          // tiles per expert: pairs of 128-row blocks, or single blocks
+      pair_prefix[e] = run;
+      const int mt = tile_prefix[e + 1] - tile_prefix[e];
+      run += kPair ? (mt + 1) >> 1 : mt;
+    }
     pair_prefix[n_experts] = run;
   }
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
-  cluster_sync_all();
+  if (kPair) cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
   const int total_tiles = pair_prefix[n_experts] * n_blocks_n;
@@ -159,31 +185,38 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
       Ring rd;
       for (; ok;) {
         const int tile = rd.next(bars, is_peer, abort_flag, status);
-        rd.done(bars, true);
+        rd.template done<kPair>(bars, true);
         if (tile < 0) break;
         TileCoord tc;
         if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-        const int row0 = padded_offsets[tc.expert] + tc.m_block * (2 * BM) + (int)rank * BM;
+        const int row0 = padded_offsets[tc.expert] + tc.m_block * kRowsPerTile + (int)rank * BM;
         const int n0 = tc.n_block * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
-          const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);
-          if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), 2 * (A_STAGE + PB_STAGE));
-          tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * BKB, row0, full);
-          tma_load_3d_pair(smem_u32(smem_b + stage * PB_STAGE), &tm_b, kb * BKB, n0, tc.expert, full);
+          if (kPair) {
+            const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);
+            if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), 2 * (A_STAGE + B_STAGE));
+            tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * BKB, row0, full);
+            tma_load_3d_pair(smem_u32(smem_b + stage * B_STAGE), &tm_b, kb * BKB, n0, tc.expert, full);
+          } else {
+            const uint32_t full = smem_u32(&bars->full[stage]);
+            mbar_expect_tx(full, A_STAGE + B_STAGE);
+            tma_load_2d(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * BKB, row0, full);
+            tma_load_3d(smem_u32(smem_b + stage * B_STAGE), &tm_b, kb * BKB, n0, tc.expert, full);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1 && lane == 0 && !is_peer) {
       // ---------------------------------------------------------------- MMA issuer (leader CTA)
-      constexpr uint32_t idesc = make_idesc_e4m3(2 * BM, BN);
+      constexpr uint32_t idesc = make_idesc_e4m3(kRowsPerTile, BN);
       int stage = 0; uint32_t phase = 0;
       int pb = 0; uint32_t pb_phase = 0;
       bool ok = true;
       Ring rd;
       for (; ok;) {
         const int tile = rd.next(bars, false, abort_flag, status);
-        rd.done(bars, true);
+        rd.template done<kPair>(bars, true);
         if (tile < 0) break;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&bars->part_empty[pb]), pb_phase ^ 1u, abort_flag, status)) { ok = false; break; }
@@ -191,12 +224,19 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(pb * BN);
           const uint64_t adesc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE));
-          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * PB_STAGE));
+          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * B_STAGE));
 #pragma unroll
-          for (int k4 = 0; k4 < BKB / 32; ++k4)          // 32 e4m3 elements of K per MMA
-            tc_mma_f8_pair(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, k4 != 0 ? 1u : 0u);
-          tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);
-          tc_commit_pair_both(smem_u32(&bars->part_full[pb]), 3);
+          for (int k4 = 0; k4 < BKB / 32; ++k4) {        // 32 e4m3 elements of K per MMA
+            if (kPair) tc_mma_f8_pair(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, k4 != 0 ? 1u : 0u);
+            else tc_mma_f8(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, k4 != 0 ? 1u : 0u);
+          }
+          if (kPair) {
+            tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);
+            tc_commit_pair_both(smem_u32(&bars->part_full[pb]), 3);
+          } else {
+            tc_commit(smem_u32(&bars->empty[stage]));
+            tc_commit(smem_u32(&bars->part_full[pb]));
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
           if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
         }
@@ -209,9 +249,9 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
         int t = atomicAdd(tile_counter, 1);
         if (t >= total_tiles) t = -1;
         bars->sched_tile[slot] = t;
-        st_shared_cluster_u32(mapa(smem_u32(&bars->sched_tile[slot]), 1), (uint32_t)t);
+        if (kPair) st_shared_cluster_u32(mapa(smem_u32(&bars->sched_tile[slot]), 1), (uint32_t)t);
         mbar_arrive(smem_u32(&bars->sched_full[slot]));
-        mbar_arrive_release_cluster(mapa(smem_u32(&bars->sched_full[slot]), 1));
+        if (kPair) mbar_arrive_release_cluster(mapa(smem_u32(&bars->sched_full[slot]), 1));
         if (t < 0) break;
         if (++slot == kRing) { slot = 0; phase ^= 1u; }
       }
@@ -233,11 +273,11 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
     for (;;) {
       const int tile = rd.next(bars, is_peer, abort_flag, status);
       __syncwarp();
-      rd.done(bars, lane == 0);
+      rd.template done<kPair>(bars, lane == 0);
       if (tile < 0) break;
       TileCoord tc;
       if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-      const int r_in_group = tc.m_block * (2 * BM) + (int)rank * BM + lane_grp * 32 + lane;
+      const int r_in_group = tc.m_block * kRowsPerTile + (int)rank * BM + lane_grp * 32 + lane;
       const bool row_ok = r_in_group < counts[tc.expert];
       const size_t grow = (size_t)(padded_offsets[tc.expert] + r_in_group);
       const float* sa_row = a_scales + grow * num_kb;
@@ -247,35 +287,63 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
 #pragma unroll
       for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
       bool ok = true;
+      // Software-pipelined promotion: the partial tile is read in four 32-column chunks per K block; the
+      // load of chunk i+1 is in flight while chunk i is multiplied and added, across K-block borders, and
+      // the scratch buffer is handed back to the MMA warp as soon as its last chunk has been read.
+#define CEP_FMA_CHUNK(V, BASE, S)                                                                   \
+  {                                                                                                  \
+    const unsigned long long s2_ = pack_f32x2(__float_as_uint(S), __float_as_uint(S));              \
+    _Pragma("unroll") for (int i = 0; i < 16; ++i)                                                  \
+        fma_f32x2(acc2[(BASE) + i], pack_f32x2((V)[2 * i], (V)[2 * i + 1]), s2_);                  \
+  }
+#ifdef CEP_EXP_NO_TMEM_LD
+#define tc_ld32(addr, v) { (v)[0] = (addr); (v)[1] = 0; }
+#endif
+#ifdef CEP_EXP_NO_FMA
+#undef CEP_FMA_CHUNK
+#define CEP_FMA_CHUNK(V, BASE, S) { acc2[(BASE)] += (V)[0] + (V)[1] + __float_as_uint(S); }
+#endif
+      uint32_t va[32], vb[32];
+      {
+        const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);
+        if (!__all_sync(0xffffffffu, got)) break;
+        tc_fence_after();
+        tc_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN + col0), va);
+        tc_wait_ld();
+      }
       for (int kb = 0; kb < num_kb; ++kb) {
         const float sa = row_ok ? __ldg(sa_row + kb) : 0.f;
         const float s0 = sa * __ldg(sw0_p + kb), s1 = sa * __ldg(sw1_p + kb);
-        const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);
-        if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-        tc_fence_after();
         const uint32_t t_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN);
-        // two 32-column loads in flight per wait; the scratch buffer is handed back to the MMA warp as
-        // soon as its last column has been read, before the final multiply-adds
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          uint32_t v0[32], v1[32];
-          tc_ld32(t_addr + (uint32_t)(g == 0 ? col0 : col1), v0);
-          tc_ld32(t_addr + (uint32_t)((g == 0 ? col0 : col1) + 32), v1);
-          tc_wait_ld();
-          if (g == 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
-          }
-          const float s = g == 0 ? s0 : s1;
-          const unsigned long long s2 = pack_f32x2(__float_as_uint(s), __float_as_uint(s));
-#pragma unroll
-          for (int i = 0; i < 16; ++i) fma_f32x2(acc2[g * 32 + i], pack_f32x2(v0[2 * i], v0[2 * i + 1]), s2);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) fma_f32x2(acc2[g * 32 + 16 + i], pack_f32x2(v1[2 * i], v1[2 * i + 1]), s2);
+        tc_ld32(t_addr + (uint32_t)(col0 + 32), vb);
+        CEP_FMA_CHUNK(va, 0, s0);
+        tc_wait_ld();
+        tc_ld32(t_addr + (uint32_t)col1, va);
+        CEP_FMA_CHUNK(vb, 16, s0);
+        tc_wait_ld();
+        tc_ld32(t_addr + (uint32_t)(col1 + 32), vb);
+        CEP_FMA_CHUNK(va, 32, s1);
+        tc_wait_ld();
+        // every column of this scratch buffer is in registers: give it back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (kPair) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
+          else mbar_arrive(smem_u32(&bars->part_empty[pb]));
         }
         if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
+        if (kb + 1 < num_kb) {
+          const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);
+          if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+          tc_fence_after();
+          tc_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN + col0), va);
+          CEP_FMA_CHUNK(vb, 48, s1);
+          tc_wait_ld();
+        } else {
+          CEP_FMA_CHUNK(vb, 48, s1);
+        }
       }
+#undef CEP_FMA_CHUNK
       if (!ok) break;
       // ---------------------------------------------------------------- epilogue from registers
       float acc[128];
@@ -340,11 +408,12 @@ grouped_gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __g
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  cluster_sync_all();
+  if (kPair) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -368,21 +437,29 @@ __global__ void pack_scales_kernel(const float* __restrict__ s_gate, const float
 }
 
 int g_clusters = -1;
+bool g_single_ready = false;
 
-cudaError_t setup(int n_sms) {
-  if (g_clusters >= 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_fp8_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+template <bool kPair>
+cudaError_t set_smem_attr() {
+  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_fp8_kernel<true, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Geo<kPair>::kSmemBytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(grouped_gemm_fp8_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  return cudaFuncSetAttribute(grouped_gemm_fp8_kernel<false, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Geo<kPair>::kSmemBytes);
+}
+
+cudaError_t setup_pair(int n_sms) {
+  if (g_clusters >= 0) return cudaSuccess;
+  cudaError_t e = set_smem_attr<true>();
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.gridDim = dim3(n_sms & ~1, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = kSmemBytes; cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.dynamicSmemBytes = Geo<true>::kSmemBytes; cfg.attrs = attr; cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_fp8_pair_kernel<true>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_fp8_kernel<true, true>, &cfg);
   if (e != cudaSuccess) return e;
   g_clusters = n;
   return cudaSuccess;
@@ -398,38 +475,57 @@ cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const
   return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_fp8_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                                 const float* a_scales, const float* b_scales, void* out, float* out_scales,
-                                 const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s, int64_t* launches) {
-  cudaError_t e = setup(n_sms);
-  if (e != cudaSuccess) return e;
-  if (g_clusters < 1) return cudaErrorNotSupported;
-  int n_blocks_n = (p.N + BN - 1) / BN;
-  int n_out_cols = p.swiglu ? p.N / 2 : p.N;
-  int clusters = max_pair_tiles < g_clusters ? max_pair_tiles : g_clusters;
-  if (clusters < 1) return cudaSuccess;
-  int num_kb = p.K / BKB;
-  int n_experts = p.n_experts, out_ld = p.out_ld;
-  int n_group = n_group_for(n_blocks_n, BN, p.K, 1);
+template <bool kSwiglu, bool kPair>
+static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, const CUtensorMap& b, int num_kb, int n_blocks_n,
+                              int n_group, int n_experts, int n_out_cols, int out_ld, const float* a_scales,
+                              const float* b_scales, void* out, float* out_scales, const LayoutPtrs& lp, int32_t* counter) {
+  return cudaLaunchKernelEx(cfg, grouped_gemm_fp8_kernel<kSwiglu, kPair>, a, b, num_kb, n_blocks_n, n_group, n_experts,
+                            n_out_cols, out_ld, a_scales, b_scales, kSwiglu ? (uint8_t*)out : (uint8_t*)nullptr,
+                            kSwiglu ? out_scales : (float*)nullptr, kSwiglu ? (__nv_bfloat16*)nullptr : (__nv_bfloat16*)out,
+                            (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
+                            counter, lp.status);
+}
+
+// pair != 0: CTA pairs on 256x256 tiles (the weight operand map must have a 128-row box, max_tiles counts pair
+// tiles); pair == 0: one CTA per 128x256 tile (256-row box, max_tiles counts single tiles).
+cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                            const float* a_scales, const float* b_scales, void* out, float* out_scales,
+                            const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches) {
+  cudaError_t e;
+  int ctas;
+  if (pair) {
+    e = setup_pair(n_sms);
+    if (e != cudaSuccess) return e;
+    if (g_clusters < 1) return cudaErrorNotSupported;
+    ctas = 2 * (max_tiles < g_clusters ? max_tiles : g_clusters);
+  } else {
+    if (!g_single_ready) {
+      e = set_smem_attr<false>();
+      if (e != cudaSuccess) return e;
+      g_single_ready = true;
+    }
+    ctas = max_tiles < n_sms ? max_tiles : n_sms;
+  }
+  if (ctas < 1) return cudaSuccess;
+  const int n_blocks_n = (p.N + BN - 1) / BN;
+  const int n_out_cols = p.swiglu ? p.N / 2 : p.N;
+  const int num_kb = p.K / BKB;
+  const int n_group = n_group_for(n_blocks_n, BN, p.K, 1);
   int32_t* counter = lp.sched + (p.swiglu ? 0 : 1);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.gridDim = dim3(2 * clusters, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[0].val.clusterDim.x = pair ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(ctas, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = pair ? Geo<true>::kSmemBytes : Geo<false>::kSmemBytes;
+  cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
-  if (p.swiglu)
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_fp8_pair_kernel<true>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols,
-                           out_ld, a_scales, b_scales, (uint8_t*)out, out_scales, (__nv_bfloat16*)nullptr,
-                           (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
-                           counter, lp.status);
-  else
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_fp8_pair_kernel<false>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols,
-                           out_ld, a_scales, b_scales, (uint8_t*)nullptr, (float*)nullptr, (__nv_bfloat16*)out,
-                           (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
-                           counter, lp.status);
+#define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, p.out_ld, \
+                                                  a_scales, b_scales, out, out_scales, lp, counter)
+  if (p.swiglu) e = pair ? CEP_FP8_LAUNCH(true, true) : CEP_FP8_LAUNCH(true, false);
+  else e = pair ? CEP_FP8_LAUNCH(false, true) : CEP_FP8_LAUNCH(false, false);
+#undef CEP_FP8_LAUNCH
   *launches += 1;
   return e;
 }

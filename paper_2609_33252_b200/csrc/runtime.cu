@@ -200,15 +200,16 @@ int launch_invocation(cep_plan* p) {
       CUDA_TRY(p, launch_gemm_simt(g1, sl.xp, p->w13p, sl.act, sl.lp, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
       CUDA_TRY(p, launch_gemm_simt(g2, sl.act, p->w2p, sl.y, sl.lp, st, &p->launches));
-    } else if (c.gemm_impl == CEP_GEMM_TCGEN05 && fp8) {
+    } else if (fp8) {
+      const int pair = c.gemm_impl == CEP_GEMM_TCGEN05 ? 1 : 0;
       const int bn = gemm_tile_cols();
-      const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
-      const long long t1 = pair_bound * ((g1.N + bn - 1) / bn), t2 = pair_bound * ((g2.N + bn - 1) / bn);
-      CUDA_TRY(p, launch_gemm_fp8_pair(g1, sl.tm_a1, p->tm_b1, sl.xp_scales, p->s13p, sl.act, sl.act_scales, sl.lp,
-                                       (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
+      const long long m_bound = pair ? (m_tiles_bound + groups + 1) / 2 : m_tiles_bound;
+      const long long t1 = m_bound * ((g1.N + bn - 1) / bn), t2 = m_bound * ((g2.N + bn - 1) / bn);
+      CUDA_TRY(p, launch_gemm_fp8(g1, pair, sl.tm_a1, p->tm_b1, sl.xp_scales, p->s13p, sl.act, sl.act_scales, sl.lp,
+                                  (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
-      CUDA_TRY(p, launch_gemm_fp8_pair(g2, sl.tm_a2, p->tm_b2, sl.act_scales, p->s2p, sl.y, nullptr, sl.lp,
-                                       (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
+      CUDA_TRY(p, launch_gemm_fp8(g2, pair, sl.tm_a2, p->tm_b2, sl.act_scales, p->s2p, sl.y, nullptr, sl.lp,
+                                  (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
     } else if (c.gemm_impl == CEP_GEMM_TCGEN05) {
       const int bn = gemm_tile_cols();
       const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
@@ -269,8 +270,8 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   *out = nullptr;
   if (!workspace) return fail(nullptr, CEP_ERR_ARG, "workspace is NULL");
   if (cfg->dtype == CEP_FP8_E4M3_BLOCK128) {
-    if (cfg->gemm_impl != CEP_GEMM_TCGEN05)
-      return fail(nullptr, CEP_ERR_UNSUPPORTED, "block-scaled fp8 runs on the CTA-pair tensor-core kernel only");
+    if (cfg->gemm_impl == CEP_GEMM_SIMT)
+      return fail(nullptr, CEP_ERR_UNSUPPORTED, "block-scaled fp8 runs on the tensor-core kernels only");
     if (cfg->hidden % 256) return fail(nullptr, CEP_ERR_ARG, "fp8 needs hidden to be a multiple of 256");
   }
   Layout L = make_layout(*cfg);

@@ -22,12 +22,13 @@ def load(layer, inp):
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
 
 
+@pytest.mark.parametrize("impl", [cep.CEP_GEMM_TCGEN05, cep.CEP_GEMM_TCGEN05_1CTA], ids=["pair", "1cta"])
 @pytest.mark.parametrize("cfg", [FP8_TINY, FP8_MID], ids=["tiny", "mid"])
-def test_fp8_matches_mirrored_oracle_and_layout_is_bit_exact(cfg):
+def test_fp8_matches_mirrored_oracle_and_layout_is_bit_exact(cfg, impl):
     host = wl.make_inputs(cfg)
     ref = oracle.from_inputs(host)                         # mirror of the intermediate re-quantisation is on for fp8
     inp = to_device(host)
-    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl)
     load(layer, inp)
     out, n_inv = run_layer(inp, layer, local_pairs=True)
     assert n_inv == 1
@@ -46,14 +47,15 @@ def test_fp8_matches_mirrored_oracle_and_layout_is_bit_exact(cfg):
     layer.close()
 
 
-def test_fp8_chunked_equals_one_shot_bitwise():
+@pytest.mark.parametrize("impl", [cep.CEP_GEMM_TCGEN05, cep.CEP_GEMM_TCGEN05_1CTA], ids=["pair", "1cta"])
+def test_fp8_chunked_equals_one_shot_bitwise(impl):
     cfg = FP8_MID
     inp = to_device(wl.make_inputs(cfg))
-    sync = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    sync = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl)
     load(sync, inp)
     one, _ = run_layer(inp, sync)
     for rep in range(3):
-        asy = make_layer(cfg, mode=cep.CEP_MODE_ASYNC, n_streams=2)
+        asy = make_layer(cfg, mode=cep.CEP_MODE_ASYNC, n_streams=2, gemm_impl=impl)
         load(asy, inp)
         two, n_inv = run_layer(inp, asy, order=[2, 0, 1])
         assert n_inv == 3
