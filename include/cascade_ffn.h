@@ -103,8 +103,9 @@ typedef struct {
   int32_t n_streams;           /* S >= 1 compute streams / scratch slots (round-robin)          */
   int64_t threshold_pairs;     /* theta: ready local (token, expert) pairs per invocation       */
   int32_t gemm_impl;           /* cep_gemm_impl                                                 */
-  int32_t debug_checks;        /* nonzero: kernels bounds-check every index and record, never
-                                  trap, on violation                                            */
+  int32_t debug_checks;        /* reserved, set to 0: the checks that exist (expert ids in range,
+                                  rows inside the scratch slot, tile-ring values) are always on
+                                  and record in the status word instead of trapping             */
   int32_t profile_kernels;     /* nonzero: record CUDA events between the kernels of every
                                   invocation so ffn_query can report per-kernel device times    */
   int32_t reserved_;           /* set to 0                                                      */
@@ -262,6 +263,14 @@ CEP_API int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens, in
 CEP_API int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n,
                           int32_t n_group, int32_t tile, int32_t* expert, int32_t* m_block,
                           int32_t* n_block);
+/*
+ * Test hook for failure detection (no counterpart in the paper).  Every wait inside the kernels is
+ * bounded; this launches, on `stream`, one thread block that waits with the same routine on a barrier
+ * nothing signals.  After limit_ms (1..1000) the wait gives up, the device status word records it and the
+ * kernel exits normally.  Call between ffn_begin and combine and pass the same stream to combine:
+ * ffn_status() then returns CEP_ERR_DEVICE_TIMEOUT, and the next layer call starts clean.
+ */
+CEP_API int cep_debug_wait_timeout(cep_plan* plan, int32_t limit_ms, void* stream);
 CEP_API int cep_debug_schedule(const int64_t* pairs, int32_t n_chunks, int32_t mode, int64_t theta,
                        int32_t* invocation_of_chunk);
 

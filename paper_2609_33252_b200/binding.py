@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout"]
 
 
 class CepConfig(ctypes.Structure):
@@ -88,6 +88,7 @@ def load_library(build_if_missing: bool = True):
         "cep_last_error": (ctypes.c_char_p, [vp]),
         "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
         "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
+        "cep_debug_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -206,6 +207,10 @@ def moe_plan_destroy(plan):
 def cep_last_error(plan=None) -> str:
     m = lib().cep_last_error(plan)
     return m.decode() if m else ""
+
+
+def cep_debug_wait_timeout(plan, limit_ms: int, stream=None):
+    _check(lib().cep_debug_wait_timeout(plan, limit_ms, _stream_handle(stream)), plan)
 
 
 def cep_debug_decode_tile(tile_prefix, n_blocks_n: int, tile: int, n_group: int = 0):

@@ -433,7 +433,29 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
   }
 }
 
+// Probe of the bounded-wait path: one CTA waits, with the same wait routine the GEMM kernels use, on a
+// barrier that nothing ever arrives on.  The wait gives up after limit_ns, records the timeout in the status
+// word and the kernel exits normally (no trap, the context stays usable).
+__global__ void wait_probe_kernel(unsigned long long limit_ns, int32_t* __restrict__ status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool got = mbar_wait_limit(smem_u32(&bar), 0u, &abort_flag, status, limit_ns);
+  if (got && threadIdx.x == 0) atomicExch(&status[kStDetail], 0xBAD);   // cannot happen: nobody arrives
+}
+
 }  // namespace
+
+cudaError_t launch_wait_probe(unsigned long long limit_ns, int32_t* status, cudaStream_t s, int64_t* launches) {
+  wait_probe_kernel<<<1, 64, 0, s>>>(limit_ns, status);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -12,6 +12,8 @@ struct alignas(64) GemmTensorMap { unsigned long long opaque[16]; };
 // entry point is unavailable, -2 when the driver rejects the description.
 int make_operand_map(GemmTensorMap* out, const void* base, int elt_bytes, int K, long long rows, int n_batch,
                      int box_rows);
+// One CTA that waits limit_ns on a barrier nobody signals, then records the timeout in status (test hook).
+cudaError_t launch_wait_probe(unsigned long long limit_ns, int32_t* status, cudaStream_t s, int64_t* launches);
 int gemm_tile_rows();
 int gemm_tile_cols();
 

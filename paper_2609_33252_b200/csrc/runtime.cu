@@ -531,6 +531,17 @@ int moe_plan_destroy(cep_plan* p) {
   return CEP_OK;
 }
 
+int cep_debug_wait_timeout(cep_plan* p, int32_t limit_ms, void* stream) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->layer_open) return fail(p, CEP_ERR_STATE, "cep_debug_wait_timeout needs an open layer call");
+  if (limit_ms < 1 || limit_ms > 1000) return fail(p, CEP_ERR_ARG, "limit_ms must be in 1..1000");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));          // after this call's status reset
+  CUDA_TRY(p, launch_wait_probe((unsigned long long)limit_ms * 1000000ull,
+                                reinterpret_cast<int32_t*>(p->ws + p->L.status), st, &p->launches));
+  return CEP_OK;
+}
+
 int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts, int32_t n_blocks_n, int32_t n_group,
                           int32_t tile, int32_t* expert, int32_t* m_block, int32_t* n_block) {
   if (!tile_prefix || n_experts <= 0 || !expert || !m_block || !n_block) return CEP_ERR_ARG;

@@ -242,6 +242,32 @@ def test_error_paths():
     assert e.value.code == -3
 
 
+def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
+    # failure detection without a fault: a wait that nothing satisfies runs out after its limit, the kernel
+    # exits normally, the host reads CEP_ERR_DEVICE_TIMEOUT, and the next layer call is clean and correct
+    import time
+    cfg = wl.CONFIGS["tiny"]
+    host = wl.make_inputs(cfg)
+    inp = to_device(host)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    load(layer, inp)
+    out = torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
+    cep.ffn_begin(layer.plan, out, cfg.T, 1)
+    cep.ffn_submit_chunk(layer.plan, 0, 0, cfg.T, inp.x, None, inp.topk_ids, inp.topk_w)
+    t0 = time.perf_counter()
+    cep.cep_debug_wait_timeout(layer.plan, 200)
+    cep.combine(layer.plan)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert 0.15 < waited < 5.0
+    assert cep.ffn_status(layer.plan) == -7
+    assert "bounded wait" in cep.cep_last_error(layer.plan)
+    check_close(out, oracle.from_inputs(host), "layer call that carried the probe")   # the real work still ran
+    out2, _ = run_layer(inp, layer)                                                     # status was reset
+    check_close(out2, oracle.from_inputs(host), "after a timeout")
+    layer.close()
+
+
 def test_kernel_launch_counter_counts_our_kernels():
     cfg = wl.CONFIGS["tiny"]
     inp = to_device(wl.make_inputs(cfg))
