@@ -406,6 +406,7 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   if (n_tokens < 0 || token_offset < 0) return fail(p, CEP_ERR_ARG, "negative n_tokens or token_offset");
   if ((long long)token_offset + n_tokens > p->n_tokens_total) return fail(p, CEP_ERR_CAPACITY, "chunk %d covers tokens beyond n_tokens_total", chunk_id);
   if (n_tokens > 0 && (!tokens || !topk_ids || !topk_weights)) return fail(p, CEP_ERR_ARG, "a chunk pointer is NULL");
+  if (reinterpret_cast<uintptr_t>(tokens) % 16) return fail(p, CEP_ERR_ARG, "chunk tokens must be 16-byte aligned");
   const bool fp8 = p->cfg.dtype == CEP_FP8_E4M3_BLOCK128;
   if (fp8 && n_tokens > 0 && !token_scales) return fail(p, CEP_ERR_ARG, "fp8 chunk without token_scales");
   const int64_t bound = (int64_t)n_tokens * p->cfg.top_k;
