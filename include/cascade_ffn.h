@@ -161,6 +161,26 @@ CEP_API int moe_load_weights(cep_plan* plan, const void* w_gate, const void* w_u
 CEP_API int ffn_begin(cep_plan* plan, void* out, int32_t n_tokens_total, int32_t n_chunks_expected);
 
 /*
+ * Optional, between ffn_begin and the first ffn_submit_chunk: `addend` [device] bf16 [n_tokens_total, H] in
+ * token order is added to every output row (fp32, before the single rounding).  This is the shared expert's
+ * output: the combine result "is added to the shared-expert output" (Appendix "Output return and combine").
+ * The rows of a chunk's tokens must be complete on that chunk's stream when the chunk is submitted.  NULL
+ * (the default after ffn_begin) adds nothing.
+ */
+CEP_API int ffn_set_addend(cep_plan* plan, const void* addend);
+
+/*
+ * Router step that precedes the path (benchmark definition; the paper does not describe its router):
+ * softmax over all experts, keep the top_k most probable, renormalise over those.  Needs no plan.
+ *   logits        [device] fp32 [n_tokens, n_experts_global], n_experts_global <= 1024
+ *   topk_ids      [device] out int32 [n_tokens, top_k]  slots in descending probability, ties to the lower id
+ *   topk_weights  [device] out fp32 [n_tokens, top_k]   softmax over the selected logits (sums to 1)
+ * Enqueued on `stream`.
+ */
+CEP_API int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts_global, int32_t top_k,
+                      int32_t* topk_ids, float* topk_weights, void* stream);
+
+/*
  * A replica's routed tokens have arrived (Section 3.2: per-replica completion signal).
  *   chunk_id       0..n_chunks_expected-1, each exactly once, any order
  *   token_offset   first token (row of `out`) this chunk covers

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route"]
 
 
 class CepConfig(ctypes.Structure):
@@ -89,6 +89,8 @@ def load_library(build_if_missing: bool = True):
         "cep_debug_decode_tile": (ctypes.c_int, [vp, i32, i32, i32, i32] + [ctypes.POINTER(i32)] * 3),
         "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
         "cep_debug_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
+        "ffn_set_addend": (ctypes.c_int, [vp, vp]),
+        "moe_route": (ctypes.c_int, [vp, i32, i32, i32, vp, vp, vp]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -149,6 +151,16 @@ def moe_load_weights(plan, w_gate, w_up, w_down, s_gate, s_up, s_down, packed, s
 
 def ffn_begin(plan, out, n_tokens_total: int, n_chunks_expected: int):
     _check(lib().ffn_begin(plan, out.data_ptr(), n_tokens_total, n_chunks_expected), plan)
+
+
+def ffn_set_addend(plan, addend):
+    _check(lib().ffn_set_addend(plan, _dptr(addend)), plan)
+
+
+def moe_route(logits, top_k: int, topk_ids, topk_weights, stream=None):
+    n_tokens, n_experts_global = logits.shape
+    _check(lib().moe_route(logits.data_ptr(), n_tokens, n_experts_global, top_k, topk_ids.data_ptr(),
+                           topk_weights.data_ptr(), _stream_handle(stream)))
 
 
 def ffn_submit_chunk(plan, chunk_id: int, token_offset: int, n_tokens: int, tokens, token_scales, topk_ids,
@@ -270,10 +282,12 @@ class MoELayer:
     def load_weights(self, w_gate, w_up, w_down, s_gate=None, s_up=None, s_down=None, stream=None):
         moe_load_weights(self.plan, w_gate, w_up, w_down, s_gate, s_up, s_down, self.packed, stream)
 
-    def run(self, out, chunks, order=None, streams=None, stream=None, n_local_pairs=None):
+    def run(self, out, chunks, order=None, streams=None, stream=None, n_local_pairs=None, addend=None):
         """chunks: list of (token_offset, x, x_scale, ids, w).  Returns the number of invocations."""
         n_tok = sum(c[1].shape[0] for c in chunks)
         ffn_begin(self.plan, out, n_tok, len(chunks))
+        if addend is not None:
+            ffn_set_addend(self.plan, addend)
         order = list(range(len(chunks))) if order is None else order
         for c in order:
             off, x, xs, ids, w = chunks[c]

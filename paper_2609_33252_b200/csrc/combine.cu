@@ -1,7 +1,9 @@
 // Top-k weighted combine + unpermute (Appendix "Output return and combine"): every routed
 // contribution is weighted by its routing coefficient exactly once and accumulated at its
 // token; results are written in token order.  Slots are accumulated in ascending slot
-// order in fp32 and rounded to bf16 once.  Tokens with no local expert get exact zeros.
+// order in fp32 and rounded to bf16 once.  Tokens with no local expert get exact zeros.  An optional addend
+// row (the shared expert's output for the token: "the result is added to the shared-expert output") is added
+// in fp32 after the routed contributions, before the single rounding.
 #include <cuda_bf16.h>
 
 #include "cep_common.h"
@@ -23,7 +25,8 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4& v, floa
 
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int32_t* __restrict__ row_of_pair,
-               const __nv_bfloat16* __restrict__ y, __nv_bfloat16* __restrict__ out) {
+               const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restrict__ addend,
+               __nv_bfloat16* __restrict__ out) {
   __shared__ int32_t s_rows[32];
   __shared__ float s_w[32];
   const int t = blockIdx.x;
@@ -37,6 +40,7 @@ combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int3
   __syncthreads();
   const int n_vec = H >> 3;
   uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(batch.chunk[c].token_offset + tl) * H);
+  const uint4* add = addend ? reinterpret_cast<const uint4*>(addend + (size_t)(batch.chunk[c].token_offset + tl) * H) : nullptr;
   for (int v = threadIdx.x; v < n_vec; v += kThreads) {
     float acc[8];
 #pragma unroll
@@ -58,6 +62,7 @@ combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int3
       const int row = s_rows[j];
       if (row >= 0) fma_bf16x8(acc, __ldcs(reinterpret_cast<const uint4*>(y + (size_t)row * H) + v), s_w[j]);
     }
+    if (add) fma_bf16x8(acc, __ldg(add + v), 1.0f);
     uint4 o;
     __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
@@ -69,10 +74,11 @@ combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int3
 }  // namespace
 
 cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, const void* y,
-                           void* out, cudaStream_t s, int64_t* launches) {
+                           const void* addend, void* out, cudaStream_t s, int64_t* launches) {
   if (batch.n_tokens == 0) return cudaSuccess;
   combine_kernel<<<batch.n_tokens, kThreads, 0, s>>>(batch, cfg.top_k, cfg.hidden, lp.row_of_pair,
                                                      static_cast<const __nv_bfloat16*>(y),
+                                                     static_cast<const __nv_bfloat16*>(addend),
                                                      static_cast<__nv_bfloat16*>(out));
   *launches += 1;
   return cudaGetLastError();

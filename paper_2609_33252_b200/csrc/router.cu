@@ -1,0 +1,67 @@
+// Router step in front of the routed-expert path (the benchmark's definition: softmax over all experts,
+// keep the k most probable, renormalise over those k; the paper itself does not describe its router).
+// One warp per token.  Selection is by logit (softmax is monotone), ties go to the lower expert id, slots are
+// in descending probability.  The renormalised weights are the softmax over the k selected logits, so the
+// full softmax denominator is never needed.  HBM-bound: T*E_g*4 bytes read, T*k*8 written.
+#include "cep_common.h"
+
+namespace cep {
+namespace {
+
+constexpr int kMaxPerLane = 32;          // E_g <= 1024
+
+__global__ void __launch_bounds__(256)
+route_kernel(const float* __restrict__ logits, int T, int E_g, int k, int32_t* __restrict__ ids,
+             float* __restrict__ weights) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= T) return;
+  const float* row = logits + (size_t)warp * E_g;
+  float v[kMaxPerLane];
+  const int per_lane = (E_g + 31) >> 5;
+#pragma unroll
+  for (int i = 0; i < kMaxPerLane; ++i) {
+    const int e = i * 32 + lane;                       // coalesced: consecutive lanes, consecutive experts
+    v[i] = (i < per_lane && e < E_g) ? __ldg(row + e) : -INFINITY;
+  }
+  float sel_logit = 0.f, first = 0.f, denom = 0.f;
+  int sel_id = 0;
+  for (int j = 0; j < k; ++j) {
+    // lane-local best (lowest index wins ties because i ascends and the comparison is strict)
+    float best = -INFINITY; int best_e = 0x7fffffff;
+#pragma unroll
+    for (int i = 0; i < kMaxPerLane; ++i) {
+      const int e = i * 32 + lane;
+      if (i < per_lane && v[i] > best) { best = v[i]; best_e = e; }
+    }
+    // warp argmax on (value desc, id asc)
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+      const int oe = __shfl_xor_sync(0xffffffffu, best_e, off);
+      if (ob > best || (ob == best && oe < best_e)) { best = ob; best_e = oe; }
+    }
+    if (j == 0) first = best;
+    const float p = __expf(best - first);              // best <= first: no overflow
+    denom += p;
+    if (lane == j) { sel_logit = p; sel_id = best_e; } // lane j keeps slot j (k <= 32)
+    if ((best_e & 31) == lane) {                       // owner removes it from further rounds
+#pragma unroll
+      for (int i = 0; i < kMaxPerLane; ++i) if (i == (best_e >> 5)) v[i] = -INFINITY;
+    }
+  }
+  if (lane < k) {
+    ids[(size_t)warp * k + lane] = sel_id;
+    weights[(size_t)warp * k + lane] = sel_logit / denom;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_route(const float* logits, int T, int E_g, int k, int32_t* ids, float* weights, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int warps_per_block = 8;
+  route_kernel<<<(T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(logits, T, E_g, k, ids, weights);
+  return cudaGetLastError();
+}
+
+}  // namespace cep

@@ -141,7 +141,7 @@ struct cep_plan {
   float* s13p; float* s2p;                      // fp8: packed weight scales
   GemmTensorMap tm_b1, tm_b2;
   // current layer call
-  void* out; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
+  void* out; const void* addend; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
   std::vector<char> chunk_seen;
   std::vector<PendingChunk> pending;
   int64_t pending_pairs;
@@ -229,7 +229,7 @@ int launch_invocation(cep_plan* p) {
                                       p->n_sms, st, &p->launches));
     }
     if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[2], st));
-    CUDA_TRY(p, launch_combine(batch, c, sl.lp, sl.y, p->out, st, &p->launches));
+    CUDA_TRY(p, launch_combine(batch, c, sl.lp, sl.y, p->addend, p->out, st, &p->launches));
   }
   CUDA_TRY(p, cudaEventRecord(iv.done, st));
   p->inv.push_back(iv);
@@ -283,7 +283,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   p->err[0] = 0; p->launches = 0;
   p->have_weights = p->layer_open = p->flushed = p->readback_pending = p->ever_closed = false;
   p->host_status = nullptr; p->begin_evt = p->readback_evt = p->weights_evt = nullptr;
-  p->out = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
+  p->out = nullptr; p->addend = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
   int dev = 0;
 #define PLAN_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
     fail(nullptr, CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); moe_plan_destroy(p); return CEP_ERR_CUDA; } } while (0)
@@ -387,7 +387,7 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   if (p->readback_pending) CUDA_TRY(p, cudaStreamWaitEvent(s0, p->readback_evt, 0));
   CUDA_TRY(p, cudaMemsetAsync(p->ws + p->L.status, 0, kStWords * sizeof(int32_t), s0));
   CUDA_TRY(p, cudaEventRecord(p->begin_evt, s0));
-  p->out = out; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
+  p->out = out; p->addend = nullptr; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
   p->n_submitted = 0; p->tokens_submitted = 0;
   p->chunk_seen.assign(n_chunks_expected, 0);
   p->pending.clear(); p->pending_pairs = 0; p->inv.clear();
@@ -424,6 +424,25 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   p->tokens_submitted += n_tokens;
   if (should_launch(p->cfg.mode, p->pending_pairs, (int)p->pending.size(), p->cfg.threshold_pairs))
     return launch_invocation(p);
+  return CEP_OK;
+}
+
+int ffn_set_addend(cep_plan* p, const void* addend) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_set_addend before ffn_begin");
+  if (p->n_submitted > 0) return fail(p, CEP_ERR_STATE, "ffn_set_addend after the first chunk was submitted");
+  if (addend && reinterpret_cast<uintptr_t>(addend) % 16) return fail(p, CEP_ERR_ARG, "addend must be 16-byte aligned");
+  p->addend = addend;
+  return CEP_OK;
+}
+
+int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts_global, int32_t top_k, int32_t* topk_ids,
+              float* topk_weights, void* stream) {
+  if (!logits || !topk_ids || !topk_weights) return fail(nullptr, CEP_ERR_ARG, "a router pointer is NULL");
+  if (n_tokens < 0 || n_experts_global <= 0 || n_experts_global > 1024 || top_k <= 0 || top_k > 32 || top_k > n_experts_global)
+    return fail(nullptr, CEP_ERR_ARG, "router needs 0 < top_k <= min(32, n_experts_global) and n_experts_global <= 1024");
+  cudaError_t e = launch_route(logits, n_tokens, n_experts_global, top_k, topk_ids, topk_weights, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail(nullptr, CEP_ERR_CUDA, "router launch failed: %s", cudaGetErrorString(e));
   return CEP_OK;
 }
 
