@@ -278,3 +278,37 @@ def test_kernel_launch_counter_counts_our_kernels():
     run_layer(inp, layer)
     assert cep.cep_kernel_launches(layer.plan) - before == 2 * 7   # 4 layout + 2 GEMM + 1 combine per invocation
     layer.close()
+
+
+# ------------------------------------------------------------------ limits of the configuration space
+def test_many_experts_and_wide_top_k():
+    # the largest expert count the plan accepts, most experts empty; then the widest top-k
+    T, H, I = 600, 256, 128
+    for E_global, E_local, k in [(1024, 1024, 4), (64, 40, 32)]:
+        host = edge_inputs(T, k, E_global, E_local, H, I, distinct_ids(T, k, E_global, 11), seed=3)
+        ref = oracle.from_inputs(host)
+        inp = to_device(host)
+        layer = make_layer(host.cfg, mode=cep.CEP_MODE_SYNC)
+        load(layer, inp)
+        out, _ = run_layer(inp, layer)
+        assert_layout_matches(layer, 0, batch_ids(host, [0]), E_local)
+        check_close(out, ref, "E=%d k=%d" % (E_local, k))
+        layer.close()
+
+
+def test_more_chunks_than_one_invocation_holds_and_empty_chunks():
+    # 40 chunks (some empty) under Sync: a batch is launched early when it holds 32 chunks
+    sizes = [7] * 20 + [0, 0, 13] + [5] * 17
+    T = sum(sizes)
+    cfg = wl.MoEConfig("chunks40", 0, T=T, H=256, I=128, E_global=8, E_local=8, k=2, chunks=tuple(sizes))
+    host = wl.make_inputs(cfg)
+    ref = oracle.from_inputs(host)
+    inp = to_device(host)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, n_streams=2)
+    load(layer, inp)
+    out, n_inv = run_layer(inp, layer)
+    assert n_inv == 2                                        # 32 chunks, then the remaining 8 at the flush
+    assert cep.ffn_query(layer.plan, 0).n_chunks == 32 and cep.ffn_query(layer.plan, 1).n_chunks == 8
+    assert_layout_matches(layer, 1, batch_ids(host, list(range(32, 40))), cfg.E_local)
+    check_close(out, ref, "40 chunks")
+    layer.close()
