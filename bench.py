@@ -251,9 +251,12 @@ def main():
 
     dt = cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16
     layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
-                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, profile_kernels=1,
-                         gemm_impl=args.gemm_impl)
+                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, gemm_impl=args.gemm_impl)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+    # a second plan that records events between the kernels: per-kernel device times, outside the timed region
+    prof_layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
+                              mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1, gemm_impl=args.gemm_impl)
+    prof_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     torch.cuda.synchronize()
     out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
     chunks = [(o, inp.x[o:o + n], None if inp.x_scale is None else inp.x_scale[o:o + n], inp.topk_ids[o:o + n],
@@ -291,11 +294,11 @@ def main():
     launches = cep.cep_kernel_launches(layer.plan) - launches0
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
     # per-kernel times: a few more steps, each followed by a sync and a query (outside the timed region)
-    for _ in range(min(args.steps, 5)):
-        step()
+    for _ in range(min(args.steps, 5) + 1):
+        prof_layer.run(out, chunks, n_local_pairs=ch_pairs)
         torch.cuda.synchronize()
-        for i in range(cep.ffn_num_invocations(layer.plan)):
-            info = cep.ffn_query(layer.plan, i)
+        for i in range(cep.ffn_num_invocations(prof_layer.plan)):
+            info = cep.ffn_query(prof_layer.plan, i)
             for k_ in kern:
                 kern[k_].append(getattr(info, k_))
     clocks = sampler.stop() if rank == 0 else None
@@ -348,6 +351,7 @@ def main():
     if rank == 0 and not args.no_stream and cfg.n_chunks > 1:
         stream_report = stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, ms * 1e-3, args)
 
+    prof_layer.close()
     if rank != 0:
         layer.close()
         if dist is not None:

@@ -46,6 +46,37 @@ struct LayoutPtrs {
   int32_t* sched;             // [2] tile counters of the two GEMMs of an invocation (zeroed by the scan kernel)
 };
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of an invocation is launched with programmatic stream serialization: it may be scheduled
+// while its predecessor in the stream is still draining, so launch latency and block scheduling overlap the
+// predecessor's tail.  Each thread first waits for the predecessor grid to complete (its memory is then
+// visible), and only then lets the successor be scheduled.  Launched without the attribute both are no-ops.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, int cluster_x,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.attrs = attr; cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------- tile scheduling arithmetic
 // Linear tile index -> (expert, m_block, n_block).  Tiles are expert-major.  Inside an expert the n
 // blocks are taken in chunks of `n_group` (the last chunk may be shorter); a chunk is swept over all

@@ -29,6 +29,7 @@ combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int3
                __nv_bfloat16* __restrict__ out) {
   __shared__ int32_t s_rows[32];
   __shared__ float s_w[32];
+  pdl_enter();
   const int t = blockIdx.x;
   int c = 0;
   while (c + 1 < batch.n_chunks && t >= batch.chunk[c + 1].token_base) ++c;
@@ -76,12 +77,10 @@ combine_kernel(const __grid_constant__ BatchDesc batch, int k, int H, const int3
 cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, const void* y,
                            const void* addend, void* out, cudaStream_t s, int64_t* launches) {
   if (batch.n_tokens == 0) return cudaSuccess;
-  combine_kernel<<<batch.n_tokens, kThreads, 0, s>>>(batch, cfg.top_k, cfg.hidden, lp.row_of_pair,
-                                                     static_cast<const __nv_bfloat16*>(y),
-                                                     static_cast<const __nv_bfloat16*>(addend),
-                                                     static_cast<__nv_bfloat16*>(out));
   *launches += 1;
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, dim3(batch.n_tokens), dim3(kThreads), 0, s, 1, batch, cfg.top_k, cfg.hidden,
+                    (const int32_t*)lp.row_of_pair, static_cast<const __nv_bfloat16*>(y),
+                    static_cast<const __nv_bfloat16*>(addend), static_cast<__nv_bfloat16*>(out));
 }
 
 }  // namespace cep

@@ -109,6 +109,7 @@ grouped_gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_
                          const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
                          int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_enter();
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + kStages * A_STAGE;
@@ -279,6 +280,7 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
                               const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
                               int32_t* __restrict__ tile_counter, int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_enter();
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + kPairStages * A_STAGE;
@@ -536,11 +538,13 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& 
   int32_t* counter = lp.sched + (p.swiglu ? 0 : 1);     // zeroed by this invocation's scan kernel
   __nv_bfloat16* o = (__nv_bfloat16*)out;
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.gridDim = dim3(2 * clusters, 1, 1); cfg.blockDim = dim3(kPairThreads, 1, 1);
-  cfg.dynamicSmemBytes = kPairSmemBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.dynamicSmemBytes = kPairSmemBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
   if (p.swiglu)

@@ -124,6 +124,7 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
                              const int32_t* __restrict__ padded_offsets, int32_t* __restrict__ tile_counter,
                              int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_enter();
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr int kStages = Geo<kPair>::kStages, B_STAGE = Geo<kPair>::B_STAGE;
   constexpr int kRowsPerTile = kPair ? 2 * BM : BM;
@@ -513,12 +514,14 @@ cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap&
   const int n_group = n_group_for(n_blocks_n, BN, p.K, 1);
   int32_t* counter = lp.sched + (p.swiglu ? 0 : 1);
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = pair ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.gridDim = dim3(ctas, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = pair ? Geo<true>::kSmemBytes : Geo<false>::kSmemBytes;
-  cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
 #define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, p.out_ld, \

@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kThreads)
 hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global, int32_t* __restrict__ seg_hist,
             int32_t* __restrict__ status) {
   extern __shared__ int32_t sh[];
+  pdl_enter();
   for (int e = threadIdx.x; e < E; e += kThreads) sh[e] = 0;
   __syncthreads();
   const int n_pairs = batch.n_tokens * k;
@@ -50,6 +51,7 @@ scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: ro
             int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ padded_offsets,
             int32_t* __restrict__ tile_prefix, int32_t* __restrict__ sched) {
   __shared__ int32_t s_cnt[1024];
+  pdl_enter();
   if (threadIdx.x < 2) sched[threadIdx.x] = 0;   // tile counters of this invocation's two GEMMs
   __shared__ int32_t s_off[1025], s_pad[1025];
   const int e = threadIdx.x;
@@ -94,6 +96,7 @@ rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t
             int32_t* __restrict__ row_of_pair, int32_t* __restrict__ pair_of_row, int cap_rows,
             int32_t* __restrict__ status) {
   extern __shared__ int32_t sh[];              // [kWarps][E] running row cursor per warp and expert
+  pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < kWarps * E; i += kThreads) sh[i] = 0;
   __syncthreads();
@@ -144,6 +147,7 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
                     const int32_t* __restrict__ row_of_pair, const int32_t* __restrict__ counts,
                     const int32_t* __restrict__ padded_offsets, int32_t* __restrict__ pair_of_row,
                     uint8_t* __restrict__ xp, float* __restrict__ xp_scales, int cap_rows) {
+  pdl_enter();
   const int n_vec = row_bytes >> 4;
   if ((int)blockIdx.x >= batch.n_tokens) {       // padding rows of expert e
     const int e = blockIdx.x - batch.n_tokens;
@@ -202,20 +206,24 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
                           float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, int64_t* launches) {
   const int k = cfg.top_k, E = cfg.n_experts_local;
   if (n_seg < 1) n_seg = 1;
-  hist_kernel<<<n_seg, kThreads, E * sizeof(int32_t), s>>>(batch, k, E, cfg.n_experts_global, lp.block_base,
-                                                           lp.status);
-  scan_kernel<<<1, 1024, 0, s>>>(n_seg, E, lp.block_base, lp.counts, lp.offsets, lp.padded_offsets,
-                                 lp.tile_prefix, lp.sched);
-  rank_kernel<<<n_seg, kThreads, kWarps * E * sizeof(int32_t), s>>>(batch, k, E, lp.block_base, lp.row_of_pair,
-                                                                   lp.pair_of_row, cap_rows, lp.status);
+  cudaError_t err;
+  err = launch_pdl(hist_kernel, dim3(n_seg), dim3(kThreads), E * sizeof(int32_t), s, 1, batch, k, E, cfg.n_experts_global,
+                   lp.block_base, lp.status);
+  if (err != cudaSuccess) return err;
+  err = launch_pdl(scan_kernel, dim3(1), dim3(1024), 0, s, 1, n_seg, E, lp.block_base, lp.counts, lp.offsets,
+                   lp.padded_offsets, lp.tile_prefix, lp.sched);
+  if (err != cudaSuccess) return err;
+  err = launch_pdl(rank_kernel, dim3(n_seg), dim3(kThreads), kWarps * E * sizeof(int32_t), s, 1, batch, k, E,
+                   (const int32_t*)lp.block_base, lp.row_of_pair, lp.pair_of_row, cap_rows, lp.status);
+  if (err != cudaSuccess) return err;
   const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128;
   const int row_bytes = cfg.hidden * (fp8 ? 1 : 2);
   const int n_scale = fp8 ? cfg.hidden / kQuantBlock : 0;
-  scatter_rows_kernel<4><<<batch.n_tokens + E, kThreads, 0, s>>>(
-      batch, k, E, row_bytes, n_scale, lp.row_of_pair, lp.counts, lp.padded_offsets, lp.pair_of_row,
-      static_cast<uint8_t*>(xp), fp8 ? xp_scales : nullptr, cap_rows);
+  err = launch_pdl(scatter_rows_kernel<4>, dim3(batch.n_tokens + E), dim3(kThreads), 0, s, 1, batch, k, E, row_bytes, n_scale,
+                   (const int32_t*)lp.row_of_pair, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
+                   lp.pair_of_row, static_cast<uint8_t*>(xp), fp8 ? xp_scales : (float*)nullptr, cap_rows);
   *launches += 4;
-  return cudaGetLastError();
+  return err;
 }
 
 }  // namespace cep
