@@ -189,9 +189,9 @@ def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
         case = {"tau": tau, "last_arrival_ms": max(arr) * 1e3}
         for name, _, _, _ in modes:
             ts, ninv = [], 0
-            for rep in range(6):
+            for rep in range(13):                  # 3 warm-up + 10 timed
                 dt, ninv = run_with_arrivals(layers[name], out, chunks, arr, ch_pairs, rstreams)
-                if rep >= 2:
+                if rep >= 3:
                     ts.append(dt)
             case[name] = {"completion_ms": statistics.median(ts) * 1e3, "min_ms": min(ts) * 1e3, "invocations": ninv}
         report["cases"].append(case)
