@@ -35,9 +35,17 @@ hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global,
   const int p0 = blockIdx.x * kSegPairs;
   const int p1 = min(p0 + kSegPairs, n_pairs);
   bool bad = false;
-  for (int p = p0 + threadIdx.x; p < p1; p += kThreads) {
-    const int e = load_pair_id(batch, k, p);
-    if (e < 0 || e >= E_global) bad = true;
+  constexpr int kPerThread = kSegPairs / kThreads;
+  int ids[kPerThread];
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {          // independent loads first: one memory latency, not eight
+    const int p = p0 + i * kThreads + threadIdx.x;
+    ids[i] = p < p1 ? load_pair_id(batch, k, p) : E;   // E: in range, not local, counted nowhere
+  }
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int e = ids[i];
+    if (e < 0 || e >= E_global) { if (p0 + i * kThreads + (int)threadIdx.x < p1) bad = true; }
     else if (e < E) atomicAdd(&sh[e], 1);
   }
   if (bad) atomicOr(&status[kStBadRouting], 1);
@@ -56,12 +64,16 @@ scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: ro
   __shared__ int32_t s_off[1025], s_pad[1025];
   const int e = threadIdx.x;
   int total = 0;
-  if (e < E) {
-    for (int s = 0; s < n_seg; ++s) {
-      const int c = seg_hist[(size_t)s * E + e];
-      seg_hist[(size_t)s * E + e] = total;      // exclusive prefix over segments
-      total += c;
+  if (e < E) {                                  // loads only, eight in flight: the stores come in the second pass
+    int s = 0;
+    for (; s + 8 <= n_seg; s += 8) {
+      int c[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) c[u] = seg_hist[(size_t)(s + u) * E + e];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) total += c[u];
     }
+    for (; s < n_seg; ++s) total += seg_hist[(size_t)s * E + e];
   }
   s_cnt[e] = (e < E) ? total : 0;
   __syncthreads();
@@ -80,8 +92,17 @@ scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: ro
     offsets[e] = s_off[e];
     padded_offsets[e] = s_pad[e];
     tile_prefix[e] = s_pad[e] / kRowAlign;
-    const int base = s_pad[e];
-    for (int s = 0; s < n_seg; ++s) seg_hist[(size_t)s * E + e] += base;
+    // histogram -> first row of each (segment, expert): exclusive prefix over the segments on top of the group start
+    int run = s_pad[e];
+    int s = 0;
+    for (; s + 8 <= n_seg; s += 8) {
+      int c[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) c[u] = seg_hist[(size_t)(s + u) * E + e];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { seg_hist[(size_t)(s + u) * E + e] = run; run += c[u]; }
+    }
+    for (; s < n_seg; ++s) { const int c = seg_hist[(size_t)s * E + e]; seg_hist[(size_t)s * E + e] = run; run += c; }
   }
   if (e == 0) {
     offsets[E] = s_off[E];
@@ -104,11 +125,19 @@ rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t
   constexpr int kPerWarp = kSegPairs / kWarps;
   const int w0 = blockIdx.x * kSegPairs + warp * kPerWarp;
   int32_t* mine = sh + warp * E;
-  // pass 1: this warp's count per expert
-  for (int it = 0; it < kPerWarp; it += 32) {
-    const int p = w0 + it + lane;
+  // this lane's ids for both passes, loaded once with independent loads
+  int my_ids[kPerWarp / 32];
+#pragma unroll
+  for (int i = 0; i < kPerWarp / 32; ++i) {
+    const int p = w0 + i * 32 + lane;
     int e = -2;
     if (p < n_pairs) { e = load_pair_id(batch, k, p); if (e < 0 || e >= E) e = -1; }
+    my_ids[i] = e;
+  }
+  // pass 1: this warp's count per expert
+#pragma unroll
+  for (int it = 0; it < kPerWarp; it += 32) {
+    const int e = my_ids[it / 32];
     const unsigned m = __match_any_sync(0xffffffffu, e);
     if (e >= 0 && lane == (__ffs(m) - 1)) mine[e] += __popc(m);
     __syncwarp();
@@ -121,10 +150,10 @@ rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t
   }
   __syncthreads();
   // pass 2: rows in pair order
+#pragma unroll
   for (int it = 0; it < kPerWarp; it += 32) {
     const int p = w0 + it + lane;
-    int e = -2;
-    if (p < n_pairs) { e = load_pair_id(batch, k, p); if (e < 0 || e >= E) e = -1; }
+    const int e = my_ids[it / 32];
     const unsigned m = __match_any_sync(0xffffffffu, e);
     int row = -1;
     if (e >= 0) row = mine[e] + __popc(m & ((1u << lane) - 1u));
