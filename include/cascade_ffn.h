@@ -103,9 +103,11 @@ typedef struct {
   int32_t n_streams;           /* S >= 1 compute streams / scratch slots (round-robin)          */
   int64_t threshold_pairs;     /* theta: ready local (token, expert) pairs per invocation       */
   int32_t gemm_impl;           /* cep_gemm_impl                                                 */
-  int32_t debug_checks;        /* reserved, set to 0: the checks that exist (expert ids in range,
-                                  rows inside the scratch slot, tile-ring values) are always on
-                                  and record in the status word instead of trapping             */
+  int32_t debug_checks;        /* nonzero: every region of the workspace is followed by a 1 KiB gap
+                                  filled with a byte pattern at moe_plan (cep_debug_check_guards
+                                  verifies them).  The in-kernel checks (expert ids in range, rows
+                                  inside the scratch slot, tile-ring values) are always on and
+                                  record in the status word instead of trapping                 */
   int32_t profile_kernels;     /* nonzero: record CUDA events between the kernels of every
                                   invocation so ffn_query can report per-kernel device times    */
   int32_t reserved_;           /* set to 0                                                      */
@@ -291,6 +293,12 @@ CEP_API int cep_debug_decode_tile(const int32_t* tile_prefix, int32_t n_experts,
  * ffn_status() then returns CEP_ERR_DEVICE_TIMEOUT, and the next layer call starts clean.
  */
 CEP_API int cep_debug_wait_timeout(cep_plan* plan, int32_t limit_ms, void* stream);
+/*
+ * Out-of-bounds tripwire for plans made with debug_checks (no counterpart in the paper): synchronises
+ * the plan's streams and compares every guard gap of the workspace with the pattern written at moe_plan.
+ * n_damaged [host out] = number of gaps that changed; 0 means no kernel wrote past the end of a region.
+ */
+CEP_API int cep_debug_check_guards(cep_plan* plan, int32_t* n_damaged);
 CEP_API int cep_debug_schedule(const int64_t* pairs, int32_t n_chunks, int32_t mode, int64_t theta,
                        int32_t* invocation_of_chunk);
 

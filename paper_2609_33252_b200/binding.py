@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards"]
 
 
 class CepConfig(ctypes.Structure):
@@ -90,6 +90,7 @@ def load_library(build_if_missing: bool = True):
         "cep_debug_schedule": (ctypes.c_int, [vp, i32, i32, i64, vp]),
         "cep_debug_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
         "ffn_set_addend": (ctypes.c_int, [vp, vp]),
+        "cep_debug_check_guards": (ctypes.c_int, [vp, ctypes.POINTER(i32)]),
         "moe_route": (ctypes.c_int, [vp, i32, i32, i32, vp, vp, vp]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
@@ -219,6 +220,13 @@ def moe_plan_destroy(plan):
 def cep_last_error(plan=None) -> str:
     m = lib().cep_last_error(plan)
     return m.decode() if m else ""
+
+
+def cep_debug_check_guards(plan) -> int:
+    """Number of damaged guard gaps of a plan made with debug_checks (0 = no overrun)."""
+    n = ctypes.c_int32(-1)
+    _check(lib().cep_debug_check_guards(plan, ctypes.byref(n)), plan)
+    return n.value
 
 
 def cep_debug_wait_timeout(plan, limit_ms: int, stream=None):

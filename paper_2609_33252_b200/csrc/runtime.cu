@@ -16,6 +16,7 @@ using namespace cep;
 namespace {
 
 char g_error[256] = "";
+constexpr int kGuardByte = 0xA5;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -57,6 +58,8 @@ struct Layout {                                   // byte offsets inside the wor
       act_scales, y;                              // offsets inside a slot
   size_t total;
   int cap_rows, n_seg_max;
+  size_t guard;                                   // bytes of poisoned gap after every region (debug_checks)
+  std::vector<size_t> guard_offsets;              // offsets inside a slot of those gaps
 };
 
 int validate(const cep_config* c, const char** why) {
@@ -87,20 +90,29 @@ Layout make_layout(const cep_config& c) {
   L.n_seg_max = (int)((max_pairs + kSegPairs - 1) / kSegPairs);
   if (L.n_seg_max < 1) L.n_seg_max = 1;
   const size_t E = c.n_experts_local, A = 256;
+  L.guard = c.debug_checks ? 1024 : 0;
   size_t o = 0;
-  L.counts = o; o = align_up(o + E * 4, A);
-  L.offsets = o; o = align_up(o + (E + 1) * 4, A);
-  L.padded = o; o = align_up(o + (E + 1) * 4, A);
-  L.tile_prefix = o; o = align_up(o + (E + 1) * 4, A);
-  L.sched = o; o = align_up(o + 2 * 4, A);
-  L.block_base = o; o = align_up(o + (size_t)L.n_seg_max * E * 4, A);
-  L.row_of_pair = o; o = align_up(o + (size_t)max_pairs * 4, A);
-  L.pair_of_row = o; o = align_up(o + (size_t)L.cap_rows * 4, A);
-  L.xp = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.hidden * elt, A);
-  L.xp_scales = o; o = align_up(o + (fp8 ? (size_t)L.cap_rows * (c.hidden / kQuantBlock) * 4 : 0), A);
-  L.act = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.inter * elt, A);
-  L.act_scales = o; o = align_up(o + (fp8 ? (size_t)L.cap_rows * (c.inter / kQuantBlock) * 4 : 0), A);
-  L.y = o = align_up(o, 1024); o = align_up(o + (size_t)L.cap_rows * c.hidden * 2, 1024);
+  // every region ends on an A boundary; with debug_checks a poisoned gap follows it
+  auto region = [&](size_t& field, size_t bytes, size_t align) {
+    o = align_up(o, align);
+    field = o;
+    o = align_up(o + bytes, A);
+    if (L.guard) { L.guard_offsets.push_back(o); o += L.guard; }
+  };
+  region(L.counts, E * 4, A);
+  region(L.offsets, (E + 1) * 4, A);
+  region(L.padded, (E + 1) * 4, A);
+  region(L.tile_prefix, (E + 1) * 4, A);
+  region(L.sched, 2 * 4, A);
+  region(L.block_base, (size_t)L.n_seg_max * E * 4, A);
+  region(L.row_of_pair, (size_t)max_pairs * 4, A);
+  region(L.pair_of_row, (size_t)L.cap_rows * 4, A);
+  region(L.xp, (size_t)L.cap_rows * c.hidden * elt, 1024);
+  region(L.xp_scales, fp8 ? (size_t)L.cap_rows * (c.hidden / kQuantBlock) * 4 : 0, A);
+  region(L.act, (size_t)L.cap_rows * c.inter * elt, 1024);
+  region(L.act_scales, fp8 ? (size_t)L.cap_rows * (c.inter / kQuantBlock) * 4 : 0, A);
+  region(L.y, (size_t)L.cap_rows * c.hidden * 2, 1024);
+  o = align_up(o, 1024);
   L.slot_bytes = o;
   L.status = 0;
   L.slot0 = 1024;
@@ -335,6 +347,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     }
     p->slots.push_back(sl);
   }
+  if (L.guard) PLAN_TRY(cudaMemsetAsync(p->ws, kGuardByte, L.total, p->streams[0]));   // gaps keep this pattern
   // status word starts clean
   PLAN_TRY(cudaMemsetAsync(p->ws + L.status, 0, kStWords * sizeof(int32_t), p->streams[0]));
   PLAN_TRY(cudaEventRecord(p->begin_evt, p->streams[0]));
@@ -559,6 +572,21 @@ int cep_debug_wait_timeout(cep_plan* p, int32_t limit_ms, void* stream) {
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));          // after this call's status reset
   CUDA_TRY(p, launch_wait_probe((unsigned long long)limit_ms * 1000000ull,
                                 reinterpret_cast<int32_t*>(p->ws + p->L.status), st, &p->launches));
+  return CEP_OK;
+}
+
+int cep_debug_check_guards(cep_plan* p, int32_t* n_damaged) {
+  if (!p || !n_damaged) return fail(p, CEP_ERR_ARG, "NULL argument");
+  *n_damaged = 0;
+  if (!p->L.guard) return fail(p, CEP_ERR_STATE, "the plan was made without debug_checks: it has no guard gaps");
+  for (cudaStream_t s : p->streams) CUDA_TRY(p, cudaStreamSynchronize(s));
+  std::vector<uint8_t> host(p->L.guard);
+  for (int s = 0; s < p->cfg.n_streams; ++s)
+    for (size_t off : p->L.guard_offsets) {
+      CUDA_TRY(p, cudaMemcpy(host.data(), p->ws + p->L.slot0 + p->L.slot_bytes * s + off, p->L.guard, cudaMemcpyDeviceToHost));
+      for (uint8_t b : host)
+        if (b != kGuardByte) { *n_damaged += 1; break; }
+    }
   return CEP_OK;
 }
 

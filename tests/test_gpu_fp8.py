@@ -28,10 +28,11 @@ def test_fp8_matches_mirrored_oracle_and_layout_is_bit_exact(cfg, impl):
     host = wl.make_inputs(cfg)
     ref = oracle.from_inputs(host)                         # mirror of the intermediate re-quantisation is on for fp8
     inp = to_device(host)
-    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl, debug_checks=1)
     load(layer, inp)
     out, n_inv = run_layer(inp, layer, local_pairs=True)
     assert n_inv == 1
+    assert cep.cep_debug_check_guards(layer.plan) == 0
     want = oracle.permute(batch_ids(host, list(range(cfg.n_chunks))), cfg.E_local, align=128)
     got = cep.ffn_debug_export(layer.plan, 0, cfg.E_local, cfg.T * cfg.k)
     assert (got["counts"] == want["counts"]).all() and (got["row_of_pair"] == want["prow_of_pair"]).all()

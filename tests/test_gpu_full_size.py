@@ -45,10 +45,11 @@ def test_ep_shard_full_size(name):
     cfg = wl.CONFIGS[name]
     inp = wl.make_inputs(cfg, device="cuda", keep_logits=False)
     host = host_view(inp)
-    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, debug_checks=1)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
     out, n_inv = run_layer(inp, layer, local_pairs=True)
     assert n_inv == 1
+    assert cep.cep_debug_check_guards(layer.plan) == 0
     # integers: every count, offset and row of all T*k pairs
     want = oracle.permute(batch_ids(host, list(range(cfg.n_chunks))), cfg.E_local, align=128)
     got = cep.ffn_debug_export(layer.plan, 0, cfg.E_local, cfg.T * cfg.k)

@@ -104,12 +104,13 @@ def test_edge_cases(case, impl):
     cfg = host.cfg
     ref = oracle.from_inputs(host)
     inp = to_device(host)
-    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, gemm_impl=impl, debug_checks=1)
     load(layer, inp)
     out, n_inv = run_layer(inp, layer)
     assert n_inv == 1
     assert_layout_matches(layer, 0, batch_ids(host, list(range(cfg.n_chunks))), cfg.E_local)
     check_close(out, ref, case)
+    assert cep.cep_debug_check_guards(layer.plan) == 0         # no kernel wrote past the end of a workspace region
     none_local = (host.topk_ids >= cfg.E_local).all(dim=1)
     if none_local.any():                                   # exact zeros, written not skipped
         assert (out.cpu()[none_local].view(torch.int16) == 0).all()
@@ -312,3 +313,23 @@ def test_more_chunks_than_one_invocation_holds_and_empty_chunks():
     assert_layout_matches(layer, 1, batch_ids(host, list(range(32, 40))), cfg.E_local)
     check_close(out, ref, "40 chunks")
     layer.close()
+
+
+def test_guard_gaps_trip_when_something_writes_past_a_region():
+    cfg = wl.CONFIGS["tiny"]
+    inp = to_device(wl.make_inputs(cfg))
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, n_streams=1, debug_checks=1)
+    load(layer, inp)
+    run_layer(inp, layer)
+    assert cep.cep_debug_check_guards(layer.plan) == 0
+    # the last gap of the slot lies within its final 2 KiB: one of these two bytes is inside it
+    ws = layer.workspace
+    ws[ws.numel() - 1030] = 0
+    ws[ws.numel() - 600] = 0
+    assert cep.cep_debug_check_guards(layer.plan) >= 1
+    layer.close()
+    plain = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    with pytest.raises(cep.CepError) as e:                   # a plan without debug_checks has no gaps to check
+        cep.cep_debug_check_guards(plain.plan)
+    assert e.value.code == -2
+    plain.close()
