@@ -91,7 +91,8 @@ class ClockSampler:
 
 
 def workload_numbers(cfg, n_pairs):
-    """Algorithmic work of one step ('Algorithmic work per unit')."""
+    """Algorithmic work of one step: 6*H*I FLOP per kept (token, expert) pair; bytes per kernel as the method
+    itself must move them (each row read/written once, each touched expert's weights read once)."""
     H, I, T, E = cfg.H, cfg.I, cfg.T, cfg.E_local
     s = 2 if cfg.dtype == "bf16" else 1 + 4.0 / 128      # bytes per element (fp8: code + its share of a 1x128 scale)
     return {
@@ -275,23 +276,31 @@ def main():
     barrier()
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    launches0 = cep.cep_kernel_launches(layer.plan)
     kern = {"layout_ms": [], "gemm1_ms": [], "gemm2_ms": [], "combine_ms": []}
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-        # per-kernel device times of this step's invocations are read after the timed region;
-        # the plan keeps only the last layer call, so collect lazily below
-    ev1.record()
-    barrier()
-    total_ms = ev0.elapsed_time(ev1)
-    launches = cep.cep_kernel_launches(layer.plan) - launches0
+    bad_reasons = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+    for attempt in range(2):            # a run that saw a thermal or hardware slowdown is taken once more
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.3)
+        launches0 = cep.cep_kernel_launches(layer.plan)
+        barrier()
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        barrier()
+        total_ms = ev0.elapsed_time(ev1)
+        launches = cep.cep_kernel_launches(layer.plan) - launches0
+        timed_clocks = sampler.stop() if rank == 0 else None
+        redo = 1 if (rank == 0 and timed_clocks and bad_reasons & set(timed_clocks.get("reasons", []))) else 0
+        if dist is not None:
+            flag = torch.tensor([redo], device="cuda")
+            dist.broadcast(flag, 0)
+            redo = int(flag.item())
+        if not redo:
+            break
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
     # per-kernel times: a few more steps, each followed by a sync and a query (outside the timed region)
     for _ in range(min(args.steps, 5) + 1):
@@ -301,7 +310,9 @@ def main():
             info = cep.ffn_query(prof_layer.plan, i)
             for k_ in kern:
                 kern[k_].append(getattr(info, k_))
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = timed_clocks
+    if clocks is not None:
+        clocks["remeasured"] = attempt == 1
     ms = max_over_ranks(total_ms / args.steps, dist, "cuda")
     value = world * cfg.T / (ms * 1e-3)
 
