@@ -1,0 +1,65 @@
+"""Seeded random configurations (shapes, expert counts, chunking, modes, streams, dtypes) against the oracle:
+integers bit-exact, floats within tolerance, chunked == one-shot bitwise, guard gaps intact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_33252_b200 as cep
+from paper_2609_33252_b200 import workloads as wl
+
+from helpers import batch_ids, check_close, make_layer, run_layer, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def random_config(seed):
+    r = np.random.default_rng(1000 + seed)
+    fp8 = seed % 4 == 3
+    H = int(r.choice([256, 512, 768, 1024])) if fp8 else int(r.choice([128, 256, 384, 640, 1024]))
+    I = int(r.choice([128, 256, 384, 512]))
+    E_global = int(r.choice([1, 2, 5, 8, 24, 64, 130]))
+    E_local = int(r.integers(1, E_global + 1))
+    k = int(r.integers(1, min(8, E_global) + 1))
+    T = int(r.integers(1, 900))
+    n_chunks = int(r.integers(1, min(6, T) + 1))
+    cuts = np.sort(r.choice(np.arange(T + 1), size=n_chunks - 1, replace=True)) if n_chunks > 1 else np.array([], int)
+    sizes = np.diff(np.concatenate([[0], cuts, [T]])).astype(int).tolist()
+    cfg = wl.MoEConfig("fuzz%d" % seed, seed % 5, T=T, H=H, I=I, E_global=E_global, E_local=E_local, k=k,
+                       chunks=tuple(sizes), dtype="fp8" if fp8 else "bf16", zipf_s=float(r.choice([0.0, 1.1])))
+    mode = int(r.choice([cep.CEP_MODE_SYNC, cep.CEP_MODE_ASYNC, cep.CEP_MODE_STREAMFFN]))
+    theta = int(r.integers(0, max(2, T * k)))
+    S = int(r.integers(1, 4))
+    order = r.permutation(n_chunks).tolist()
+    return cfg, mode, theta, S, order
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_configuration(seed):
+    cfg, mode, theta, S, order = random_config(seed)
+    host = wl.make_inputs(cfg)
+    ref = oracle.from_inputs(host)
+    inp = to_device(host)
+
+    def load(layer):
+        layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+
+    sync = make_layer(cfg, mode=cep.CEP_MODE_SYNC, debug_checks=1)
+    load(sync)
+    base, n_inv = run_layer(inp, sync, local_pairs=True)
+    assert n_inv == 1
+    want = oracle.permute(batch_ids(host, list(range(cfg.n_chunks))), cfg.E_local, align=128)
+    got = cep.ffn_debug_export(sync.plan, 0, cfg.E_local, cfg.T * cfg.k)
+    for a, b in (("counts", "counts"), ("offsets", "offsets"), ("padded_offsets", "padded_offsets"),
+                 ("row_of_pair", "prow_of_pair"), ("pair_of_row", "pair_of_prow")):
+        assert (got[a] == want[b]).all(), (a, cfg)
+    check_close(base, ref, str(cfg))
+    assert cep.cep_debug_check_guards(sync.plan) == 0
+    layer = make_layer(cfg, mode=mode, theta=theta, n_streams=S, debug_checks=1)
+    load(layer)
+    pairs = [int((host.topk_ids[o:o + n] < cfg.E_local).sum()) for o, n in zip(host.chunk_offsets, cfg.chunks)]
+    out, n_inv = run_layer(inp, layer, order=order, local_pairs=True)
+    assert n_inv == len(oracle.schedule([pairs[c] for c in order], mode, theta, S, max_chunks_per_invocation=32))
+    assert torch.equal(out.view(torch.int16), base.view(torch.int16)), (cfg, mode, theta, S, order)
+    assert cep.cep_debug_check_guards(layer.plan) == 0
+    sync.close(); layer.close()
