@@ -327,8 +327,18 @@ def main():
         rstreams = [torch.cuda.Stream() for _ in chunks]
         main = torch.cuda.current_stream()
 
+        # chunks are consumed as they land (Async+streamFFN, theta = two chunks' worth of pairs) and every
+        # invocation's output rows are copied back as soon as that invocation has written them
+        e2e_theta = max(1, 2 * (sum(ch_pairs) // max(len(ch_pairs), 1)))
+        e2e_layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
+                                 mode=cep.CEP_MODE_STREAMFFN, n_streams=args.streams, threshold_pairs=e2e_theta,
+                                 gemm_impl=args.gemm_impl)
+        e2e_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+        d2h = torch.cuda.Stream()
+
         def e2e_step():
-            cep.ffn_begin(layer.plan, out, cfg.T, len(chunks))
+            cep.ffn_begin(e2e_layer.plan, out, cfg.T, len(chunks))
+            seen = 0
             for c, (o, n) in enumerate(zip(inp.chunk_offsets, cfg.chunks)):
                 st = rstreams[c]
                 st.wait_stream(main)
@@ -338,11 +348,22 @@ def main():
                     dw[o:o + n].copy_(hw[o:o + n], non_blocking=True)
                     if dxs is not None:
                         dxs[o:o + n].copy_(hxs[o:o + n], non_blocking=True)
-                cep.ffn_submit_chunk(layer.plan, c, o, n, dx[o:o + n], None if dxs is None else dxs[o:o + n],
+                cep.ffn_submit_chunk(e2e_layer.plan, c, o, n, dx[o:o + n], None if dxs is None else dxs[o:o + n],
                                      did[o:o + n], dw[o:o + n], ch_pairs[c], st)
-            cep.ffn_flush(layer.plan)
-            cep.combine(layer.plan, main)
-            hout.copy_(out, non_blocking=True)
+                if c == len(chunks) - 1:
+                    cep.ffn_flush(e2e_layer.plan)
+                # copy back the rows of every invocation launched so far (chunks are submitted in id order)
+                while seen < cep.ffn_num_invocations(e2e_layer.plan):
+                    info = cep.ffn_query(e2e_layer.plan, seen)
+                    cep.ffn_wait_invocation(e2e_layer.plan, seen, d2h)
+                    lo = inp.chunk_offsets[info.first_chunk_pos]
+                    last = info.first_chunk_pos + info.n_chunks - 1
+                    hi = inp.chunk_offsets[last] + cfg.chunks[last]
+                    with torch.cuda.stream(d2h):
+                        hout[lo:hi].copy_(out[lo:hi], non_blocking=True)
+                    seen += 1
+            cep.combine(e2e_layer.plan, main)
+            main.wait_stream(d2h)
 
         for _ in range(3):
             e2e_step()
@@ -354,7 +375,9 @@ def main():
         barrier()
         e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / args.steps, dist, "cuda")
         h2d = hx.numel() * hx.element_size() + hid.numel() * 4 + hw.numel() * 4 + (0 if hxs is None else hxs.numel() * 4)
+        e2e_layer.close()
         e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "mode": "Async+streamFFN, theta=%d pairs, per-invocation output copy-back" % e2e_theta,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": hout.numel() * 2}
 
     # ---- chunked asynchronous execution under seeded arrival offsets (rank 0 only, outside the timed step)

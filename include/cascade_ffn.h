@@ -218,6 +218,14 @@ CEP_API int combine(cep_plan* plan, void* stream);
  * CEP_OK, CEP_ERR_BAD_ROUTING or CEP_ERR_DEVICE_TIMEOUT. */
 CEP_API int ffn_status(cep_plan* plan);
 
+/*
+ * Asynchronous output return (Appendix "Output return and combine": outputs are returned asynchronously,
+ * readiness is tracked separately from the layer boundary).  Makes `stream` wait until invocation `inv` of the
+ * current layer call has written the output rows of its chunks (ffn_query tells which chunks it holds), so a
+ * caller can start consuming or copying those rows before the other invocations finish.  Does not block the host.
+ */
+CEP_API int ffn_wait_invocation(cep_plan* plan, int32_t inv, void* stream);
+
 /* Number of invocations launched in the current / last layer call. */
 CEP_API int ffn_num_invocations(const cep_plan* plan);
 

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards", "ffn_wait_invocation"]
 
 
 class CepConfig(ctypes.Structure):
@@ -81,6 +81,7 @@ def load_library(build_if_missing: bool = True):
         "combine": (ctypes.c_int, [vp, vp]),
         "ffn_status": (ctypes.c_int, [vp]),
         "ffn_num_invocations": (ctypes.c_int, [vp]),
+        "ffn_wait_invocation": (ctypes.c_int, [vp, i32, vp]),
         "ffn_query": (ctypes.c_int, [vp, i32, ctypes.POINTER(InvocationInfo)]),
         "ffn_debug_export": (ctypes.c_int, [vp, i32, vp, vp, vp, vp, vp]),
         "cep_kernel_launches": (i64, [vp]),
@@ -181,6 +182,10 @@ def combine(plan, stream=None, allow_incomplete: bool = False) -> int:
 
 def ffn_status(plan) -> int:
     return lib().ffn_status(plan)
+
+
+def ffn_wait_invocation(plan, inv: int, stream=None):
+    _check(lib().ffn_wait_invocation(plan, inv, _stream_handle(stream)), plan)
 
 
 def ffn_num_invocations(plan) -> int:

@@ -499,6 +499,13 @@ int ffn_status(cep_plan* p) {
   return CEP_OK;
 }
 
+int ffn_wait_invocation(cep_plan* p, int32_t inv, void* stream) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
+  CUDA_TRY(p, cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), p->inv[inv].done, 0));
+  return CEP_OK;
+}
+
 int ffn_num_invocations(const cep_plan* p) { return p ? (int)p->inv.size() : CEP_ERR_ARG; }
 
 int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {

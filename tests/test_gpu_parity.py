@@ -333,3 +333,38 @@ def test_guard_gaps_trip_when_something_writes_past_a_region():
         cep.cep_debug_check_guards(plain.plan)
     assert e.value.code == -2
     plain.close()
+
+
+def test_outputs_can_be_consumed_per_invocation():
+    # asynchronous output return: after waiting on one invocation only, the rows of its chunks are final
+    cfg = wl.CONFIGS["mid"]
+    host = wl.make_inputs(cfg)
+    inp = to_device(host)
+    sync = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    load(sync, inp)
+    base, _ = run_layer(inp, sync)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_ASYNC, n_streams=2)
+    load(layer, inp)
+    out = torch.full((cfg.T, cfg.H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ch = chunks_of(inp)
+    cep.ffn_begin(layer.plan, out, cfg.T, len(ch))
+    side = torch.cuda.Stream()
+    copies = []
+    for c, (off, x, xs, ids, w) in enumerate(ch):
+        cep.ffn_submit_chunk(layer.plan, c, off, x.shape[0], x, xs, ids, w)
+        info = cep.ffn_query(layer.plan, c)
+        assert info.first_chunk_pos == c and info.n_chunks == 1
+        cep.ffn_wait_invocation(layer.plan, c, side)
+        with torch.cuda.stream(side):
+            copies.append((off, x.shape[0], out[off:off + x.shape[0]].clone()))
+    side.synchronize()                                      # only the side stream: the layer is still open
+    for off, n, rows in copies:
+        assert torch.equal(rows.view(torch.int16), base[off:off + n].view(torch.int16))
+    with pytest.raises(cep.CepError) as e:
+        cep.ffn_wait_invocation(layer.plan, 99, side)
+    assert e.value.code == -1
+    cep.combine(layer.plan)
+    torch.cuda.synchronize()
+    assert cep.ffn_status(layer.plan) == 0
+    assert torch.equal(out.view(torch.int16), base.view(torch.int16))
+    sync.close(); layer.close()
