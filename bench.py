@@ -303,8 +303,11 @@ def main():
             break
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
     # per-kernel times: a few more steps, each followed by a sync and a query (outside the timed region)
-    for _ in range(min(args.steps, 5) + 1):
-        prof_layer.run(out, chunks, n_local_pairs=ch_pairs)
+    # per-kernel device times: the profiled plan runs the same number of steps back to back (same clocks and
+    # thermal state as the timed region); the plan keeps the events of its last layer call, read after a sync
+    for rep in range(3):
+        for _ in range(max(args.steps // 3, 1)):
+            prof_layer.run(out, chunks, n_local_pairs=ch_pairs)
         torch.cuda.synchronize()
         for i in range(cep.ffn_num_invocations(prof_layer.plan)):
             info = cep.ffn_query(prof_layer.plan, i)
@@ -397,10 +400,11 @@ def main():
     ffn_tflops = work["flops"] / ((g1_ms + g2_ms) * 1e-3) / 1e12
     g1_tflops = work["gemm1_flops"] / (g1_ms * 1e-3) / 1e12
     g2_tflops = work["gemm2_flops"] / (g2_ms * 1e-3) / 1e12
-    # burst peak for a short timed region at full clocks, sustained peak once the run is long enough
-    # to sit under the power cap (clock well below maximum, or more than a second of back-to-back steps)
+    # burst peak for a short timed region at full clocks; sustained peak once the steps run under the power cap
+    # (cap reported active, clock well below maximum, or more than a second of back-to-back steps)
     sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
-    sustained = (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
+    capped = "sw_power_cap" in ((clocks or {}).get("reasons") or [])
+    sustained = capped or (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
     peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     nominal_tf = NOMINAL_BF16_TFLOPS
     if cfg.dtype == "fp8":          # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2)
