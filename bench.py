@@ -276,7 +276,7 @@ def main():
     barrier()
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
 
-    kern = {"layout_ms": [], "gemm1_ms": [], "gemm2_ms": [], "combine_ms": []}
+    kern = {"layout_ms": [], "gemm1_ms": [], "gemm2_ms": [], "combine_ms": [], "index_ms": [], "scatter_ms": []}
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     bad_reasons = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
     for attempt in range(2):            # a run that saw a thermal or hardware slowdown is taken once more
@@ -420,6 +420,9 @@ def main():
     kernels = {
         "layout": {"ms": med["layout_ms"], "GB/s": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9,
                    "frac_of_hbm": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "index (hist+scan+rank)": {"ms": med["index_ms"]},
+        "scatter_rows": {"ms": med["scatter_ms"], "GB/s": work["layout_bytes"] / (med["scatter_ms"] * 1e-3) / 1e9,
+                         "frac_of_hbm": work["layout_bytes"] / (med["scatter_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "gemm1": {"ms": g1_ms, "TFLOP/s": g1_tflops},
         "gemm2": {"ms": g2_ms, "TFLOP/s": g2_tflops, "frac": g2_tflops / peak_tf},
         "combine": {"ms": med["combine_ms"], "GB/s": work["combine_bytes"] / (med["combine_ms"] * 1e-3) / 1e9,

@@ -125,6 +125,8 @@ typedef struct {
   float gemm1_ms;              /* gate/up GEMM with fused SiLU*up      else < 0)                 */
   float gemm2_ms;              /* down GEMM                                                     */
   float combine_ms;            /* weighted combine + unpermute                                  */
+  float index_ms;              /* histogram + scan + rank (the integer part of layout_ms)       */
+  float scatter_ms;            /* row scatter (the payload part of layout_ms)                   */
 } cep_invocation_info;
 
 /* Bytes of device workspace a plan with this configuration needs.  [host] out. */

@@ -41,7 +41,7 @@ class InvocationInfo(ctypes.Structure):
                 ("stream_index", ctypes.c_int32), ("n_tokens", ctypes.c_int32),
                 ("pairs_bound", ctypes.c_int64), ("elapsed_ms", ctypes.c_float),
                 ("layout_ms", ctypes.c_float), ("gemm1_ms", ctypes.c_float), ("gemm2_ms", ctypes.c_float),
-                ("combine_ms", ctypes.c_float)]
+                ("combine_ms", ctypes.c_float), ("index_ms", ctypes.c_float), ("scatter_ms", ctypes.c_float)]
 
 
 class CepError(RuntimeError):

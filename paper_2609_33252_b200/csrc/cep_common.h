@@ -129,8 +129,10 @@ struct GemmProblem {
   int is_fp8;
 };
 
+// after_index: optional event recorded between the index kernels (hist, scan, rank) and the row scatter
 cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
-                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, int64_t* launches);
+                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
+                          int64_t* launches);
 cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp,
                            const void* y, const void* addend, void* out, cudaStream_t s, int64_t* launches);
 cudaError_t launch_route(const float* logits, int T, int E_g, int k, int32_t* ids, float* weights, cudaStream_t s);

@@ -232,7 +232,8 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
 }  // namespace
 
 cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
-                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, int64_t* launches) {
+                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
+                          int64_t* launches) {
   const int k = cfg.top_k, E = cfg.n_experts_local;
   if (n_seg < 1) n_seg = 1;
   cudaError_t err;
@@ -245,6 +246,7 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
   err = launch_pdl(rank_kernel, dim3(n_seg), dim3(kThreads), kWarps * E * sizeof(int32_t), s, 1, batch, k, E,
                    (const int32_t*)lp.block_base, lp.row_of_pair, lp.pair_of_row, cap_rows, lp.status);
   if (err != cudaSuccess) return err;
+  if (after_index) { err = cudaEventRecord(after_index, s); if (err != cudaSuccess) return err; }
   const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128;
   const int row_bytes = cfg.hidden * (fp8 ? 1 : 2);
   const int n_scale = fp8 ? cfg.hidden / kQuantBlock : 0;

@@ -32,7 +32,7 @@ struct Invocation {
   int first_pos, n_chunks, slot, n_tokens;
   int64_t pairs_bound;
   cudaEvent_t start, done;
-  cudaEvent_t mark[3];          // after layout, after GEMM1, after GEMM2 (profile_kernels)
+  cudaEvent_t mark[4];          // after layout, after GEMM1, after GEMM2, after the index kernels (profile_kernels)
   bool profiled;
 };
 
@@ -146,7 +146,7 @@ struct cep_plan {
   std::vector<cudaEvent_t> ready_evt;           // per chunk position
   std::vector<Invocation> inv;
   std::vector<cudaEvent_t> inv_start, inv_done; // pools, one per possible invocation
-  std::vector<cudaEvent_t> inv_mark;            // 3 per possible invocation (profile_kernels)
+  std::vector<cudaEvent_t> inv_mark;            // 4 per possible invocation (profile_kernels)
   cudaEvent_t begin_evt, readback_evt, weights_evt;
   bool have_weights, layer_open, flushed, readback_pending, ever_closed;
   uint8_t* w13p; uint8_t* w2p;
@@ -194,14 +194,15 @@ int launch_invocation(cep_plan* p) {
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->weights_evt, 0));
   for (size_t i = 0; i < p->pending.size(); ++i) CUDA_TRY(p, cudaStreamWaitEvent(st, p->ready_evt[first_pos + (int)i], 0));
   Invocation iv{first_pos, batch.n_chunks, slot_i, tok, p->pending_pairs, p->inv_start[idx], p->inv_done[idx],
-                {nullptr, nullptr, nullptr}, false};
+                {nullptr, nullptr, nullptr, nullptr}, false};
   const bool prof = c.profile_kernels != 0 && tok > 0;
-  if (prof) { for (int m = 0; m < 3; ++m) iv.mark[m] = p->inv_mark[3 * idx + m]; iv.profiled = true; }
+  if (prof) { for (int m = 0; m < 4; ++m) iv.mark[m] = p->inv_mark[4 * idx + m]; iv.profiled = true; }
   CUDA_TRY(p, cudaEventRecord(iv.start, st));
   if (tok > 0) {
     const long long n_pairs = (long long)tok * c.top_k;
     const int n_seg = (int)((n_pairs + kSegPairs - 1) / kSegPairs);
-    CUDA_TRY(p, launch_layout(batch, c, sl.lp, sl.xp, sl.xp_scales, p->L.cap_rows, n_seg, st, &p->launches));
+    CUDA_TRY(p, launch_layout(batch, c, sl.lp, sl.xp, sl.xp_scales, p->L.cap_rows, n_seg, st, prof ? iv.mark[3] : nullptr,
+                              &p->launches));
     if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[0], st));
     const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
     const long long groups = c.n_experts_local < n_pairs ? c.n_experts_local : n_pairs;
@@ -317,7 +318,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     PLAN_TRY(cudaEventCreate(&e)); p->inv_start.push_back(e);
     PLAN_TRY(cudaEventCreate(&e)); p->inv_done.push_back(e);
     if (cfg->profile_kernels)
-      for (int m = 0; m < 3; ++m) { PLAN_TRY(cudaEventCreate(&e)); p->inv_mark.push_back(e); }
+      for (int m = 0; m < 4; ++m) { PLAN_TRY(cudaEventCreate(&e)); p->inv_mark.push_back(e); }
   }
   const bool fp8 = cfg->dtype == CEP_FP8_E4M3_BLOCK128;
   const int elt = fp8 ? 1 : 2;
@@ -514,12 +515,14 @@ int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {
   const Invocation& iv = p->inv[inv];
   info->n_chunks = iv.n_chunks; info->first_chunk_pos = iv.first_pos; info->stream_index = iv.slot;
   info->n_tokens = iv.n_tokens; info->pairs_bound = iv.pairs_bound; info->elapsed_ms = -1.f;
-  info->layout_ms = info->gemm1_ms = info->gemm2_ms = info->combine_ms = -1.f;
+  info->layout_ms = info->gemm1_ms = info->gemm2_ms = info->combine_ms = info->index_ms = info->scatter_ms = -1.f;
   if (cudaEventQuery(iv.done) == cudaSuccess) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, iv.start, iv.done) == cudaSuccess) info->elapsed_ms = ms;
     if (iv.profiled) {
       if (cudaEventElapsedTime(&ms, iv.start, iv.mark[0]) == cudaSuccess) info->layout_ms = ms;
+      if (cudaEventElapsedTime(&ms, iv.start, iv.mark[3]) == cudaSuccess) info->index_ms = ms;
+      if (cudaEventElapsedTime(&ms, iv.mark[3], iv.mark[0]) == cudaSuccess) info->scatter_ms = ms;
       if (cudaEventElapsedTime(&ms, iv.mark[0], iv.mark[1]) == cudaSuccess) info->gemm1_ms = ms;
       if (cudaEventElapsedTime(&ms, iv.mark[1], iv.mark[2]) == cudaSuccess) info->gemm2_ms = ms;
       if (cudaEventElapsedTime(&ms, iv.mark[2], iv.done) == cudaSuccess) info->combine_ms = ms;
