@@ -91,7 +91,7 @@ typedef enum {
 #define CEP_ROW_ALIGN 128                  /* expert groups start on multiples of the GEMM tile */
 
 typedef struct {
-  int32_t hidden;              /* H; multiple of 128 (bf16: multiple of 64)                     */
+  int32_t hidden;              /* H; multiple of 128 (fp8: multiple of 256)                     */
   int32_t inter;               /* I; multiple of 128                                            */
   int32_t n_experts_global;    /* E_g                                                           */
   int32_t n_experts_local;     /* E <= E_g, at most 1024                                        */
