@@ -392,6 +392,7 @@ def main():
     if rank != 0:
         layer.close()
         if dist is not None:
+            dist.barrier()                      # rank 0 is still measuring its rank-0-only legs
             dist.destroy_process_group()
         return 0
 
@@ -454,9 +455,10 @@ def main():
                                 "sample": "%d evenly spaced tokens of the %s workload, all their local routed "
                                           "pairs, fp64, %.1f s" % (n_s, cfg.name, dt),
                                 "rel_fro_error_of_gpu_on_sample": rel}
-    print(json.dumps(line))
+    print(json.dumps(line), flush=True)
     layer.close()
     if dist is not None:
+        dist.barrier()
         dist.destroy_process_group()
     return 0
 
