@@ -15,7 +15,8 @@ Contents (each function cites the passage of the paper it restates):
                        (Section 3.2 "Launch threshold", "Multi-stream execution";
                        Section 5.4 ablation modes)
 * ``moe_forward``      the fp64 layer result (C, ``oracle_moe.c``)
-* codecs               bf16 / e4m3 decode and encode (C)
+* codecs               bf16 / e4m3 / e2m1 / ue8m0 decode and encode, the microscaling block
+                       scale rule (C)
 
 Parity pins live in ``tests/test_oracle_*.py``; nothing here is "parity unpinned".
 """
@@ -32,8 +33,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "liboracle_moe.so")
 _SRC = os.path.join(_HERE, "oracle_moe.c")
 
-F64, BF16, FP8 = 0, 1, 2
-MIRROR_FP8_ACT, MIRROR_BF16_ACT = 1, 2
+F64, BF16, FP8, MXFP4 = 0, 1, 2, 3
+MIRROR_FP8_ACT, MIRROR_BF16_ACT, MIRROR_MXFP8_ACT = 1, 2, 4
 
 
 def build(force: bool = False) -> str:
@@ -61,6 +62,14 @@ def lib():
         L.oracle_f64_to_e4m3.argtypes = [ctypes.c_double]
         L.oracle_f64_to_bf16.restype = ctypes.c_uint16
         L.oracle_f64_to_bf16.argtypes = [ctypes.c_double]
+        L.oracle_e2m1_to_f64.restype = ctypes.c_double
+        L.oracle_e2m1_to_f64.argtypes = [ctypes.c_uint8]
+        L.oracle_f64_to_e2m1.restype = ctypes.c_uint8
+        L.oracle_f64_to_e2m1.argtypes = [ctypes.c_double]
+        L.oracle_ue8m0_to_f64.restype = ctypes.c_double
+        L.oracle_ue8m0_to_f64.argtypes = [ctypes.c_uint8]
+        L.oracle_mx_scale_code.restype = ctypes.c_uint8
+        L.oracle_mx_scale_code.argtypes = [ctypes.c_float, ctypes.c_int, ctypes.c_double]
         L.oracle_silu.restype = ctypes.c_double
         L.oracle_silu.argtypes = [ctypes.c_double]
         L.oracle_num_threads.restype = ctypes.c_int
@@ -87,6 +96,24 @@ def f64_to_e4m3(x: float) -> int:
 
 def f64_to_bf16(x: float) -> int:
     return lib().oracle_f64_to_bf16(float(x))
+
+
+def e2m1_to_f64(code: int) -> float:
+    return lib().oracle_e2m1_to_f64(int(code))
+
+
+def f64_to_e2m1(x: float) -> int:
+    return lib().oracle_f64_to_e2m1(float(x))
+
+
+def ue8m0_to_f64(code: int) -> float:
+    return lib().oracle_ue8m0_to_f64(int(code))
+
+
+def mx_scale_code(amax: float, elem: str) -> int:
+    """ue8m0 code of a 32-element block whose largest magnitude is ``amax`` (binary32)."""
+    emax, top = {"e4m3": (8, 0.75), "e2m1": (2, 0.5)}[elem]
+    return lib().oracle_mx_scale_code(float(np.float32(amax)), emax, top)
 
 
 def silu(x: float) -> float:
@@ -219,7 +246,9 @@ def moe_forward(dtype: int, X, Xs, ids, w, Wg, Wgs, Wu, Wus, Wd, Wds, E_local: i
     """fp64 result of the layer for tokens ``sel`` (all tokens when None).
 
     bf16 tensors are passed as uint16 bit patterns, fp8 tensors as uint8 codes plus fp32
-    block scales, F64 tensors as float64.  Weight layouts: Wg,Wu [E,H,I]; Wd [E,I,H].
+    block scales, F64 tensors as float64.  MXFP4: X e4m3 codes with ue8m0 scales [T,H/32];
+    weights one e2m1 code per byte with ue8m0 scales [E,in/32,out].
+    Weight layouts: Wg,Wu [E,H,I]; Wd [E,I,H].
     """
     X = np.ascontiguousarray(X)
     T, H = X.shape
@@ -228,16 +257,20 @@ def moe_forward(dtype: int, X, Xs, ids, w, Wg, Wgs, Wu, Wus, Wd, Wds, E_local: i
     ids = np.ascontiguousarray(ids, dtype=np.int32)
     w = np.ascontiguousarray(w, dtype=np.float32)
     k = ids.shape[1]
-    want = {F64: np.float64, BF16: np.uint16, FP8: np.uint8}[dtype]
+    want = {F64: np.float64, BF16: np.uint16, FP8: np.uint8, MXFP4: np.uint8}[dtype]
     arrs = []
     for a in (X, Wg, Wu, Wd):
         assert a.dtype == want, (a.dtype, want)
         arrs.append(np.ascontiguousarray(a))
     X, Wg, Wu, Wd = arrs
-    scal = [None if s is None else np.ascontiguousarray(s, dtype=np.float32)
-            for s in (Xs, Wgs, Wus, Wds)]
-    if dtype == FP8:
+    sdt = np.uint8 if dtype == MXFP4 else np.float32
+    for s_ in (Xs, Wgs, Wus, Wds):
+        assert s_ is None or s_.dtype == sdt, (s_.dtype, sdt)
+    scal = [None if s is None else np.ascontiguousarray(s) for s in (Xs, Wgs, Wus, Wds)]
+    if dtype in (FP8, MXFP4):
         assert all(s is not None for s in scal)
+    if dtype == MXFP4:
+        assert scal[0].shape == (T, H // 32) and scal[1].shape == (E, H // 32, I) and scal[3].shape == (E, I // 32, H)
     if sel is None:
         sel_arr, n_sel = None, T
     else:
@@ -262,17 +295,21 @@ def from_inputs(inp, sel=None, mirror=None, nthreads=0) -> np.ndarray:
     """Run ``moe_forward`` on a ``workloads.MoEInputs`` (tensors are copied to host)."""
     import torch
     fp8 = inp.cfg.dtype == "fp8"
+    mx = inp.cfg.dtype == "mxfp4"
 
     def bits(t):
         t = t.detach().cpu().contiguous()
-        return t.view(torch.uint8).numpy() if fp8 else t.view(torch.int16).numpy().view(np.uint16)
+        return t.view(torch.uint8).numpy() if (fp8 or mx) else t.view(torch.int16).numpy().view(np.uint16)
 
     def f32(t):
-        return None if t is None else t.detach().cpu().float().contiguous().numpy()
+        if t is None:
+            return None
+        t = t.detach().cpu().contiguous()
+        return t.view(torch.uint8).numpy() if mx else t.float().numpy()
 
     if mirror is None:
-        mirror = MIRROR_FP8_ACT if fp8 else 0
-    return moe_forward(FP8 if fp8 else BF16, bits(inp.x), f32(inp.x_scale),
+        mirror = MIRROR_FP8_ACT if fp8 else (MIRROR_MXFP8_ACT if mx else 0)
+    return moe_forward(FP8 if fp8 else (MXFP4 if mx else BF16), bits(inp.x), f32(inp.x_scale),
                        inp.topk_ids.cpu().numpy(), inp.topk_w.cpu().numpy(),
                        bits(inp.w_gate), f32(inp.s_gate), bits(inp.w_up), f32(inp.s_up),
                        bits(inp.w_down), f32(inp.s_down), inp.cfg.E_local, sel=sel,

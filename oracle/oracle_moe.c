@@ -20,6 +20,13 @@
  * Parity pins (tests/test_oracle_*.py): per-token brute force in another language
  * and loop nest, dense-MLP special cases through library matmuls, closed forms of
  * silu, exhaustive codec tables.  No function here is "parity unpinned".
+ *
+ * Microscaling operands (Section 5.1: the routed-expert weights of two of the three
+ * evaluated models are MXFP4): a block of 32 consecutive elements along the contraction
+ * dimension shares one power-of-two scale stored as an 8-bit exponent (ue8m0); weights are
+ * e2m1 elements, activations e4m3 elements.  The paper gives no quantisation rule; the one
+ * taken here is "the smallest power of two that brings the block's largest magnitude
+ * inside the element range", elements rounded to nearest even.
  */
 #include <math.h>
 #include <stdint.h>
@@ -29,8 +36,8 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_F64 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2 };
-enum { ORACLE_MIRROR_FP8_ACT = 1, ORACLE_MIRROR_BF16_ACT = 2 };
+enum { ORACLE_F64 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2, ORACLE_MXFP4 = 3 };
+enum { ORACLE_MIRROR_FP8_ACT = 1, ORACLE_MIRROR_BF16_ACT = 2, ORACLE_MIRROR_MXFP8_ACT = 4 };
 
 /* ---- codecs: exact decoders and the two round-to-nearest-even encoders ---- */
 
@@ -89,6 +96,52 @@ uint16_t oracle_f64_to_bf16(double x) {
   return (uint16_t)(u >> 16);
 }
 
+/* e2m1: 1 sign, 2 exponent (bias 1), 1 mantissa bit; magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6.
+ * The code sits in the low four bits of the byte. */
+double oracle_e2m1_to_f64(uint8_t c) {
+  int s = (c >> 3) & 1, e = (c >> 1) & 3, m = c & 1;
+  double v = (e == 0) ? 0.5 * m : ldexp(1.0 + 0.5 * m, e - 1);
+  return s ? -v : v;
+}
+
+/* Round-to-nearest-even onto the e2m1 grid, saturating at +-6. */
+uint8_t oracle_f64_to_e2m1(double x) {
+  static const double grid[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+  uint8_t s = signbit(x) ? 8 : 0;
+  double a = fabs(x);
+  if (isnan(a) || a >= 6.0) return s | 7;
+  int best = 0;
+  for (int c = 1; c < 8; ++c) {
+    double d0 = fabs(a - grid[best]), d1 = fabs(a - grid[c]);
+    if (d1 < d0 || (d1 == d0 && (c & 1) == 0)) best = c;   /* ties: the code with an even mantissa */
+  }
+  return s | (uint8_t)best;
+}
+
+/* ue8m0: an unsigned power-of-two scale, value 2^(c-127); code 255 is NaN. */
+double oracle_ue8m0_to_f64(uint8_t c) {
+  if (c == 255) return NAN;
+  return ldexp(1.0, (int)c - 127);
+}
+
+/* Block scale of a microscaling block: the smallest power of two s with
+ * amax <= elem_max * s, as a ue8m0 code, where elem_max = 1.75*2^8 (e4m3, emax=8,
+ * top mantissa 0.75) or 1.5*2^2 (e2m1).  amax is taken in binary32: with biased
+ * exponent E and fraction f of amax, log2(s) = E - 127 - emax, one more when
+ * f > top mantissa.  An all-zero block gets scale 1 (code 127); the code is clamped
+ * to 0..254. */
+uint8_t oracle_mx_scale_code(float amax, int emax, double top_mantissa) {
+  if (amax == 0.0f) return 127;
+  uint32_t u;
+  memcpy(&u, &amax, 4);
+  int E = (int)((u >> 23) & 0xff);
+  double f = (double)(u & 0x7fffffu) / 8388608.0;
+  int code = E - emax + (f > top_mantissa ? 1 : 0);
+  if (code < 0) code = 0;
+  if (code > 254) code = 254;
+  return (uint8_t)code;
+}
+
 double oracle_silu(double x) { return x / (1.0 + exp(-x)); }
 
 /* ---- element access in fp64 ---- */
@@ -96,30 +149,37 @@ double oracle_silu(double x) { return x / (1.0 + exp(-x)); }
 typedef struct {
   int dtype;
   const void *data;
-  const float *scale; /* fp8 only */
+  const void *scale; /* fp8: fp32 block scales; mxfp4: ue8m0 codes */
 } tensor_t;
 
-/* activations: [T,H], fp8 scales [T,H/128] */
+/* activations: [T,H]; fp8 scales fp32 [T,H/128]; mxfp4: e4m3 codes, ue8m0 scales [T,H/32] */
 static double x_at(const tensor_t *x, int64_t H, int64_t t, int64_t h) {
   int64_t i = t * H + h;
   switch (x->dtype) {
     case ORACLE_F64: return ((const double *)x->data)[i];
     case ORACLE_BF16: return oracle_bf16_to_f64(((const uint16_t *)x->data)[i]);
+    case ORACLE_MXFP4:
+      return oracle_e4m3_to_f64(((const uint8_t *)x->data)[i]) *
+             oracle_ue8m0_to_f64(((const uint8_t *)x->scale)[t * (H / 32) + h / 32]);
     default:
       return oracle_e4m3_to_f64(((const uint8_t *)x->data)[i]) *
-             (double)x->scale[t * (H / 128) + h / 128];
+             (double)((const float *)x->scale)[t * (H / 128) + h / 128];
   }
 }
 
-/* weights: [E,R,C] row-major, fp8 scales [E,R/128,C/128] */
+/* weights: [E,R,C] row-major (R = contraction dimension); fp8 scales fp32 [E,R/128,C/128];
+ * mxfp4: one e2m1 code per byte, ue8m0 scales [E,R/32,C] (32 consecutive r share a scale) */
 static double w_at(const tensor_t *w, int64_t R, int64_t C, int64_t e, int64_t r, int64_t c) {
   int64_t i = (e * R + r) * C + c;
   switch (w->dtype) {
     case ORACLE_F64: return ((const double *)w->data)[i];
     case ORACLE_BF16: return oracle_bf16_to_f64(((const uint16_t *)w->data)[i]);
+    case ORACLE_MXFP4:
+      return oracle_e2m1_to_f64(((const uint8_t *)w->data)[i] & 15) *
+             oracle_ue8m0_to_f64(((const uint8_t *)w->scale)[(e * (R / 32) + r / 32) * C + c]);
     default:
       return oracle_e4m3_to_f64(((const uint8_t *)w->data)[i]) *
-             (double)w->scale[(e * (R / 128) + r / 128) * (C / 128) + c / 128];
+             (double)((const float *)w->scale)[(e * (R / 128) + r / 128) * (C / 128) + c / 128];
   }
 }
 
@@ -143,6 +203,23 @@ static void requant_fp8_row(double *a, int64_t I) {
   }
 }
 
+/* Re-quantisation of the intermediate for the microscaling configuration: per row and
+ * per 32-wide block, ue8m0 scale from the block's amax (rule above, e4m3 elements), code =
+ * RNE e4m3 of a/scale (a division by a power of two), value = code*scale. */
+static void requant_mxfp8_row(double *a, int64_t I) {
+  for (int64_t b = 0; b < I; b += 32) {
+    int64_t n = (I - b < 32) ? (I - b) : 32;
+    double amax = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+      double v = fabs(a[b + i]);
+      if (v > amax) amax = v;
+    }
+    double s = oracle_ue8m0_to_f64(oracle_mx_scale_code((float)amax, 8, 0.75));
+    for (int64_t i = 0; i < n; ++i)
+      a[b + i] = oracle_e4m3_to_f64(oracle_f64_to_e4m3(a[b + i] / s)) * s;
+  }
+}
+
 /*
  * The layer, for a selection of tokens.
  *   ids  [T,k] global expert ids; ids >= E_local belong to another rank and are skipped
@@ -153,9 +230,9 @@ static void requant_fp8_row(double *a, int64_t I) {
  * Returns 0, or -1 on a bad expert id (<0).
  */
 int oracle_moe_forward(int dtype, int64_t T, int64_t H, int64_t I, int64_t E_local, int64_t k,
-                       const void *X, const float *Xs, const int32_t *ids, const float *w,
-                       const void *Wg, const float *Wgs, const void *Wu, const float *Wus,
-                       const void *Wd, const float *Wds, const int64_t *sel, int64_t n_sel,
+                       const void *X, const void *Xs, const int32_t *ids, const float *w,
+                       const void *Wg, const void *Wgs, const void *Wu, const void *Wus,
+                       const void *Wd, const void *Wds, const int64_t *sel, int64_t n_sel,
                        int mirror, double *out, int nthreads) {
   tensor_t tx = {dtype, X, Xs}, tg = {dtype, Wg, Wgs}, tu = {dtype, Wu, Wus}, td = {dtype, Wd, Wds};
   int bad = 0;
@@ -191,6 +268,7 @@ int oracle_moe_forward(int dtype, int64_t T, int64_t H, int64_t I, int64_t E_loc
         }
         for (int64_t i = 0; i < I; ++i) g[i] = oracle_silu(g[i]) * u[i];   /* a = silu(g) * u */
         if (mirror & ORACLE_MIRROR_FP8_ACT) requant_fp8_row(g, I);
+        if (mirror & ORACLE_MIRROR_MXFP8_ACT) requant_mxfp8_row(g, I);
         if (mirror & ORACLE_MIRROR_BF16_ACT)
           for (int64_t i = 0; i < I; ++i) g[i] = oracle_bf16_to_f64(oracle_f64_to_bf16(g[i]));
         for (int64_t h = 0; h < H; ++h) y[h] = 0.0;

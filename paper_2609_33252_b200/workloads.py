@@ -12,7 +12,11 @@ those traces are not available, so every tensor is synthetic and seeded.
 
 Representation: all tensors are torch tensors on ``device``.  bf16 tensors are
 ``torch.bfloat16``; block-scaled fp8 tensors are a ``torch.float8_e4m3fn`` code
-tensor plus an fp32 scale tensor (``value = code * scale``).
+tensor plus an fp32 scale tensor (``value = code * scale``).  Microscaling ("mxfp4")
+configurations: activations are ``torch.float8_e4m3fn`` codes with ``uint8`` ue8m0
+scales per 1x32 block along the hidden dimension; weights are ``uint8`` tensors holding
+one e2m1 code (low four bits) per element with ``uint8`` ue8m0 scales per 32 elements of
+the input (contraction) dimension and per output column (``value = code * 2^(scale-127)``).
 """
 from __future__ import annotations
 
@@ -39,7 +43,7 @@ class MoEConfig:
     E_local: int               # experts resident on this rank: ids 0..E_local-1
     k: int                     # experts per token
     chunks: Sequence[int]      # tokens per replica chunk, in chunk-id order
-    dtype: str = "bf16"        # "bf16" | "fp8"
+    dtype: str = "bf16"        # "bf16" | "fp8" | "mxfp4"
     zipf_s: float = 0.0        # 0 => N(0,1) logits; >0 => logits biased by -s*ln(rank)
     zipf_strided: bool = False  # popularity rank strided across ranks instead of literal
     arrival_sigma: float = 0.5  # lognormal(0, sigma) arrival offsets
@@ -78,6 +82,13 @@ CONFIGS = {
                                  chunks=tuple(_equal_chunks(2048, 8)), dtype="fp8", zipf_s=1.1),
     "fp8_shard": MoEConfig("fp8_shard", 4, T=32768, H=7168, I=3072, E_global=512, E_local=64, k=8,
                            chunks=tuple(_equal_chunks(32768, 8)), dtype="fp8", zipf_s=1.1),
+    # microscaling variant of the EP shard (Section 5.1: MXFP4 routed-expert weights): same shapes and routing
+    "mxfp4_tiny": MoEConfig("mxfp4_tiny", 5, T=256, H=512, I=256, E_global=8, E_local=8, k=2,
+                            chunks=(160, 96), dtype="mxfp4"),
+    "mxfp4_shard_small": MoEConfig("mxfp4_shard_small", 5, T=2048, H=7168, I=2048, E_global=64, E_local=8, k=8,
+                                   chunks=tuple(_equal_chunks(2048, 8)), dtype="mxfp4", zipf_s=1.1),
+    "mxfp4_shard": MoEConfig("mxfp4_shard", 5, T=16384, H=7168, I=2048, E_global=256, E_local=32, k=8,
+                             chunks=tuple(_equal_chunks(16384, 8)), dtype="mxfp4", zipf_s=1.1),
 }
 
 
@@ -185,6 +196,47 @@ def quantize_blocks_128x128(w: torch.Tensor):
     return q.view(E, R, C), scale.contiguous()
 
 
+MX_BLOCK = 32
+
+
+def mx_scale_codes(amax: torch.Tensor, elem: str) -> torch.Tensor:
+    """ue8m0 code of the smallest power of two s with amax <= elem_max * s (127 for amax == 0)."""
+    emax, top = {"e4m3": (8, 0x600000), "e2m1": (2, 0x400000)}[elem]
+    bits = amax.float().contiguous().view(torch.int32)
+    code = ((bits >> 23) & 0xFF) - emax + ((bits & 0x7FFFFF) > top).to(torch.int32)
+    code = code.clamp_(0, 254)
+    return torch.where(amax == 0, torch.full_like(code, 127), code).to(torch.uint8)
+
+
+def _to_e2m1(y: torch.Tensor) -> torch.Tensor:
+    """Round-to-nearest-even of fp32 values with |y| <= 6 onto the e2m1 grid; uint8 codes."""
+    a = y.abs()
+    code = ((a > 0.25).to(torch.uint8) + (a >= 0.75).to(torch.uint8) + (a > 1.25).to(torch.uint8) +
+            (a >= 1.75).to(torch.uint8) + (a > 2.5).to(torch.uint8) + (a >= 3.5).to(torch.uint8) +
+            (a > 5.0).to(torch.uint8))
+    return code | (torch.signbit(y).to(torch.uint8) << 3)
+
+
+def quantize_mx(x: torch.Tensor, elem: str, dim: int):
+    """Microscaling quantisation of an fp32 tensor in blocks of 32 along ``dim``.
+
+    Returns (codes, scales): codes have the shape of x (``float8_e4m3fn`` for "e4m3", ``uint8``
+    with the code in the low four bits for "e2m1"); scales are uint8 ue8m0 codes with ``dim``
+    shrunk by 32.
+    """
+    x = x.float().movedim(dim, -1)
+    shp = x.shape
+    assert shp[-1] % MX_BLOCK == 0
+    xb = x.reshape(shp[:-1] + (shp[-1] // MX_BLOCK, MX_BLOCK))
+    sc = mx_scale_codes(xb.abs().amax(dim=-1), elem)
+    y = xb * torch.exp2(127.0 - sc.float())[..., None]          # exact: a power of two
+    if elem == "e4m3":
+        q = y.clamp_(-FP8_MAX, FP8_MAX).to(torch.float8_e4m3fn)
+    else:
+        q = _to_e2m1(y)
+    return q.reshape(shp).movedim(-1, dim).contiguous(), sc.movedim(-1, dim).contiguous()
+
+
 def make_arrivals(cfg: MoEConfig) -> List[float]:
     """Unitless lognormal(0, sigma) arrival offsets, one per chunk (CPU generator)."""
     g = _gen(SEED_BASE + 16 * cfg.index + 5, "cpu")
@@ -207,7 +259,23 @@ def make_inputs(cfg: MoEConfig, device="cpu", keep_logits=True) -> MoEInputs:
     H, I, E = cfg.H, cfg.I, cfg.E_local
     fp8 = cfg.dtype == "fp8"
     sg = su = sd = xs = None
-    if not fp8:
+    if cfg.dtype == "mxfp4":
+        x32 = torch.randn((cfg.T, H), generator=_gen(seed + 1, device), device=device)
+        x, xs = quantize_mx(x32, "e4m3", 1)
+        del x32
+
+        def mxweights(shape, std, sd_):
+            g = _gen(sd_, device)
+            codes = torch.empty(shape, dtype=torch.uint8, device=device)
+            scales = torch.empty((shape[0], shape[1] // MX_BLOCK, shape[2]), dtype=torch.uint8, device=device)
+            for e in range(shape[0]):
+                blk = torch.randn(tuple(shape[1:]), generator=g, device=device) * std
+                codes[e], scales[e] = quantize_mx(blk, "e2m1", 0)
+            return codes, scales
+        wg, sg = mxweights((E, H, I), H ** -0.5, seed + 2)
+        wu, su = mxweights((E, H, I), H ** -0.5, seed + 3)
+        wd, sd = mxweights((E, I, H), I ** -0.5, seed + 4)
+    elif not fp8:
         x = _randn_chunked((cfg.T, H), 1.0, _gen(seed + 1, device), device, torch.bfloat16)
         wg = _randn_chunked((E, H, I), H ** -0.5, _gen(seed + 2, device), device, torch.bfloat16)
         wu = _randn_chunked((E, H, I), H ** -0.5, _gen(seed + 3, device), device, torch.bfloat16)
