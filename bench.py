@@ -177,7 +177,7 @@ def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
     layers = {}
     for name, mode, th, S in modes:
         L = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, mode=mode,
-                         dtype=cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16,
+                         dtype=cep.DTYPE_OF[cfg.dtype],
                          n_streams=S, threshold_pairs=th, gemm_impl=args.gemm_impl)
         L.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
         layers[name] = L
@@ -250,7 +250,7 @@ def main():
     work = workload_numbers(cfg, n_pairs)
     ch_pairs = [int((inp.topk_ids[o:o + n] < cfg.E_local).sum().item()) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
 
-    dt = cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16
+    dt = cep.DTYPE_OF[cfg.dtype]
     layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
                          mode=cep.CEP_MODE_SYNC, n_streams=args.streams, gemm_impl=args.gemm_impl)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)

@@ -69,8 +69,15 @@ typedef enum {
 
 typedef enum {
   CEP_BF16 = 0,                /* bf16 activations and weights, fp32 accumulate, bf16 output    */
-  CEP_FP8_E4M3_BLOCK128 = 1    /* e4m3 codes; fp32 scales per 1x128 activation block and per
+  CEP_FP8_E4M3_BLOCK128 = 1,   /* e4m3 codes; fp32 scales per 1x128 activation block and per
                                   128x128 weight block; bf16 output                              */
+  CEP_MXFP4_E4M3 = 2           /* microscaling: MXFP4 expert weights (Section 5.1), e2m1 codes with
+                                  one ue8m0 scale (2^(s-127)) per 32 elements of the input
+                                  dimension; e4m3 activations with one ue8m0 scale per 1x32 block
+                                  along the hidden dimension; the intermediate is re-quantised the
+                                  same way (scale = the smallest power of two that brings the
+                                  block's largest magnitude to <= 448, round to nearest even);
+                                  fp32 accumulate; bf16 output                                   */
 } cep_dtype;
 
 /* Execution modes of the ablation in Section 5.4. */
@@ -91,7 +98,7 @@ typedef enum {
 #define CEP_ROW_ALIGN 128                  /* expert groups start on multiples of the GEMM tile */
 
 typedef struct {
-  int32_t hidden;              /* H; multiple of 128 (fp8: multiple of 256)                     */
+  int32_t hidden;              /* H; multiple of 128 (fp8, mxfp4: multiple of 256)              */
   int32_t inter;               /* I; multiple of 128                                            */
   int32_t n_experts_global;    /* E_g                                                           */
   int32_t n_experts_local;     /* E <= E_g, at most 1024                                        */
@@ -146,14 +153,17 @@ CEP_API int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_by
 
 /*
  * One-off weight prepack, off the hot path.  Inputs [device]:
- *   w_gate, w_up  [E, H, I]   w_down [E, I, H]     (bf16, or e4m3 codes)
- *   s_gate, s_up  [E, H/128, I/128]  s_down [E, I/128, H/128]   fp32, fp8 only, else NULL
+ *   w_gate, w_up  [E, H, I]   w_down [E, I, H]     (bf16, or e4m3 codes, or for mxfp4 one
+ *                                                   e2m1 code per byte in its low four bits)
+ *   s_gate, s_up  [E, H/128, I/128]  s_down [E, I/128, H/128]   fp32, for fp8
+ *   s_gate, s_up  [E, H/32, I]       s_down [E, I/32, H]        uint8 ue8m0, for mxfp4
+ *                 (32 consecutive elements of the input dimension share a scale); NULL for bf16
  * `packed` [device], 256-byte aligned, moe_packed_weight_bytes() long, must outlive the
  * plan's use of it.  The transposes are enqueued on `stream` (cudaStream_t); later
  * layer calls are ordered after them.
  */
 CEP_API int moe_load_weights(cep_plan* plan, const void* w_gate, const void* w_up, const void* w_down,
-                     const float* s_gate, const float* s_up, const float* s_down,
+                     const void* s_gate, const void* s_up, const void* s_down,
                      void* packed, size_t packed_bytes, void* stream);
 
 /*
@@ -189,7 +199,7 @@ CEP_API int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts_g
  *   chunk_id       0..n_chunks_expected-1, each exactly once, any order
  *   token_offset   first token (row of `out`) this chunk covers
  *   tokens         [device] bf16 [n,H]  |  e4m3 [n,H]
- *   token_scales   [device] fp32 [n,H/128] for fp8, else NULL
+ *   token_scales   [device] fp32 [n,H/128] for fp8; uint8 ue8m0 [n,H/32] for mxfp4; else NULL
  *   topk_ids       [device] int32 [n,k] global expert ids, distinct per token
  *   topk_weights   [device] fp32 [n,k]
  *   n_local_pairs  number of (token,slot) pairs with id < n_experts_local, as known from
@@ -200,7 +210,7 @@ CEP_API int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts_g
  * Returns immediately.  May launch an invocation (see cep_mode).
  */
 CEP_API int ffn_submit_chunk(cep_plan* plan, int32_t chunk_id, int32_t token_offset, int32_t n_tokens,
-                     const void* tokens, const float* token_scales, const int32_t* topk_ids,
+                     const void* tokens, const void* token_scales, const int32_t* topk_ids,
                      const float* topk_weights, int64_t n_local_pairs, void* stream);
 
 /* All tokens have arrived: launch whatever is pending regardless of theta

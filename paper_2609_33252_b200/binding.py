@@ -13,7 +13,8 @@ from typing import List, Optional, Sequence
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libcascade_ffn.so")
 
-CEP_BF16, CEP_FP8_E4M3_BLOCK128 = 0, 1
+CEP_BF16, CEP_FP8_E4M3_BLOCK128, CEP_MXFP4_E4M3 = 0, 1, 2
+DTYPE_OF = {"bf16": CEP_BF16, "fp8": CEP_FP8_E4M3_BLOCK128, "mxfp4": CEP_MXFP4_E4M3}   # workload dtype names
 CEP_MODE_SYNC, CEP_MODE_ASYNC, CEP_MODE_STREAMFFN = 0, 1, 2
 CEP_GEMM_TCGEN05, CEP_GEMM_SIMT, CEP_GEMM_TCGEN05_1CTA = 0, 1, 2
 STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ERR_WORKSPACE",

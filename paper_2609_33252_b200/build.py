@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcascade_ffn.so")
-SOURCES = ["runtime.cu", "layout.cu", "combine.cu", "prepack.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "gemm_tcgen05_fp8.cu", "router.cu"]
+SOURCES = ["runtime.cu", "layout.cu", "combine.cu", "prepack.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "gemm_tcgen05_fp8.cu", "gemm_tcgen05_mx.cu", "router.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-diag-suppress", "177"]
 

@@ -36,7 +36,7 @@ def profile(cfg: wl.MoEConfig, rows: Sequence[int] = (16, 32, 64, 128, 256, 512,
     E, k, H, I = cfg.E_local, min(cfg.k, cfg.E_local), cfg.H, cfg.I
     fp8 = cfg.dtype == "fp8"
     max_T = max(rows) * E // k
-    layer = cep.MoELayer(H, I, E, E, k, max_T, 1, dtype=cep.CEP_FP8_E4M3_BLOCK128 if fp8 else cep.CEP_BF16,
+    layer = cep.MoELayer(H, I, E, E, k, max_T, 1, dtype=cep.DTYPE_OF[cfg.dtype],
                          mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     g = torch.Generator(device=device).manual_seed(wl.SEED_BASE + 99)
@@ -47,6 +47,8 @@ def profile(cfg: wl.MoEConfig, rows: Sequence[int] = (16, 32, 64, 128, 256, 512,
         x32 = torch.randn((T, H), generator=g, device=device)
         if fp8:
             x, xs = wl.quantize_rows_1x128(x32)
+        elif cfg.dtype == "mxfp4":
+            x, xs = wl.quantize_mx(x32, "e4m3", 1)
         else:
             x, xs = x32.to(torch.bfloat16), None
         out = torch.empty((T, H), dtype=torch.bfloat16, device=device)

@@ -11,6 +11,15 @@ constexpr int kRowAlign = CEP_ROW_ALIGN;        // rows per GEMM M tile; expert 
 constexpr int kMaxChunksPerInv = CEP_MAX_CHUNKS_PER_INVOCATION;
 constexpr int kSegPairs = 2048;                 // pairs per block in the histogram / rank kernels
 constexpr int kQuantBlock = 128;                // fp8 scale block
+constexpr int kMxBlock = 32;                    // microscaling block (elements sharing a ue8m0 scale)
+// Microscaling scale factors travel in 512-byte "atoms": the scales of 128 rows x 4 consecutive 32-blocks of K,
+// byte (r%32)*16 + (r/32)*4 + kb, which is the order tcgen05.cp (32x128b.warpx4) and the block-scaled MMA
+// expect them in.  An operand of R rows and K columns has (R/128) x (K/128) atoms, K fastest.
+constexpr int kSfAtomBytes = 512;
+__host__ __device__ inline size_t sf_atom_offset(long long row, int kb32, int k128_per_row) {
+  return ((size_t)(row >> 7) * k128_per_row + (kb32 >> 2)) * kSfAtomBytes + (size_t)((row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb32 & 3));
+}
+__host__ __device__ inline bool dtype_is_bytes(int dtype) { return dtype != CEP_BF16; }   // one-byte activation codes
 
 // Device status word layout (int32 each).
 enum StatusWord { kStBadRouting = 0, kStTimeout = 1, kStBoundsViolation = 2, kStDetail = 3, kStWords = 8 };
@@ -18,7 +27,7 @@ enum StatusWord { kStBadRouting = 0, kStTimeout = 1, kStBoundsViolation = 2, kSt
 // One chunk of a batch as the kernels see it.
 struct ChunkDesc {
   const void* tokens;         // [n,H] bf16 | e4m3
-  const float* scales;        // fp8: [n,H/128]
+  const void* scales;         // fp8: fp32 [n,H/128]; mxfp4: ue8m0 bytes [n,H/32]
   const int32_t* ids;         // [n,k]
   const float* weights;       // [n,k]
   int32_t n_tokens;
@@ -126,12 +135,12 @@ struct GemmProblem {
   int swiglu;                 // 1: output column j = silu(acc[:, pair(j)]) * acc[:, pair(j)+128]
   int out_ld;                 // elements per output row
   int cap_rows;               // rows the A / output buffers hold
-  int is_fp8;
+  int is_fp8;                 // any one-byte operand format (block-scaled e4m3 or microscaling)
 };
 
 // after_index: optional event recorded between the index kernels (hist, scan, rank) and the row scatter
 cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
-                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
+                          void* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
                           int64_t* launches);
 cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp,
                            const void* y, const void* addend, void* out, cudaStream_t s, int64_t* launches);

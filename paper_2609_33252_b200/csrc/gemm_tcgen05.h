@@ -38,4 +38,18 @@ cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap&
 cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const float* s_up, const float* s_down,
                                float* s13p, float* s2p, cudaStream_t s, int64_t* launches);
 
+// Microscaling variant (e4m3 activations x packed e2m1 weights, ue8m0 scales per 32 elements of K, scaled by the
+// tensor core).  CTA pairs on 256x256 tiles.  Scale factors of both operands are read through 2-D maps over
+// their 512-byte atoms (see kSfAtomBytes); with p.swiglu the output is e4m3 codes [rows, N/2] plus their scale
+// atoms out_sf, otherwise bf16 [rows, N].
+int make_mx_weight_map(GemmTensorMap* out, const void* base, int K, long long rows, int n_batch, int box_rows);
+int make_mx_sf_map(GemmTensorMap* out, const void* base, long long n_loads, int atom_bytes);
+cudaError_t launch_gemm_mx(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
+                           const GemmTensorMap& tm_sfa, const GemmTensorMap& tm_sfb, void* out, void* out_sf,
+                           const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s, int64_t* launches);
+// codes [E,in,out] (one e2m1 code per byte) -> K-major packed nibbles; scales [E,in/32,out] -> scale atoms
+cudaError_t launch_prepack_mx(const cep_config& cfg, const void* w_gate, const void* w_up, const void* w_down,
+                              const void* s_gate, const void* s_up, const void* s_down, void* w13p, void* w2p,
+                              void* sf13p, void* sf2p, cudaStream_t s, int64_t* launches);
+
 }  // namespace cep

@@ -175,7 +175,8 @@ __global__ void __launch_bounds__(kThreads)
 scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int row_bytes, int n_scale,
                     const int32_t* __restrict__ row_of_pair, const int32_t* __restrict__ counts,
                     const int32_t* __restrict__ padded_offsets, int32_t* __restrict__ pair_of_row,
-                    uint8_t* __restrict__ xp, float* __restrict__ xp_scales, int cap_rows) {
+                    uint8_t* __restrict__ xp, uint32_t* __restrict__ xp_scales /*32-bit words: an fp32 scale, or
+                    four ue8m0 bytes*/, int sf_atoms /*scale words go to the 512-byte atom order*/, int cap_rows) {
   pdl_enter();
   const int n_vec = row_bytes >> 4;
   if ((int)blockIdx.x >= batch.n_tokens) {       // padding rows of expert e
@@ -185,7 +186,9 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
     for (int r = r0; r < r1 && r < cap_rows; ++r) {
       uint4* dst = reinterpret_cast<uint4*>(xp + (size_t)r * row_bytes);
       for (int v = threadIdx.x; v < n_vec; v += kThreads) dst[v] = make_uint4(0, 0, 0, 0);
-      if (xp_scales) for (int v = threadIdx.x; v < n_scale; v += kThreads) xp_scales[(size_t)r * n_scale + v] = 0.f;
+      if (xp_scales)
+        for (int v = threadIdx.x; v < n_scale; v += kThreads)
+          xp_scales[sf_atoms ? sf_atom_offset(r, 4 * v, n_scale) >> 2 : (size_t)r * n_scale + v] = 0u;
       if (threadIdx.x == 0) pair_of_row[r] = -1;
     }
     return;
@@ -218,12 +221,12 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
     }
   }
   if (xp_scales) {
-    const float* ss = batch.chunk[c].scales + (size_t)tl * n_scale;
+    const uint32_t* ss = static_cast<const uint32_t*>(batch.chunk[c].scales) + (size_t)tl * n_scale;
     for (int v = threadIdx.x; v < n_scale; v += kThreads) {
-      const float sv = __ldg(ss + v);
+      const uint32_t sv = __ldg(ss + v);
       for (int j = 0; j < k; ++j) {
         const int row = s_rows[j];
-        if (row >= 0) xp_scales[(size_t)row * n_scale + v] = sv;
+        if (row >= 0) xp_scales[sf_atoms ? sf_atom_offset(row, 4 * v, n_scale) >> 2 : (size_t)row * n_scale + v] = sv;
       }
     }
   }
@@ -232,7 +235,7 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
 }  // namespace
 
 cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp, void* xp,
-                          float* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
+                          void* xp_scales, int cap_rows, int n_seg, cudaStream_t s, cudaEvent_t after_index,
                           int64_t* launches) {
   const int k = cfg.top_k, E = cfg.n_experts_local;
   if (n_seg < 1) n_seg = 1;
@@ -247,12 +250,13 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
                    (const int32_t*)lp.block_base, lp.row_of_pair, lp.pair_of_row, cap_rows, lp.status);
   if (err != cudaSuccess) return err;
   if (after_index) { err = cudaEventRecord(after_index, s); if (err != cudaSuccess) return err; }
-  const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128;
-  const int row_bytes = cfg.hidden * (fp8 ? 1 : 2);
-  const int n_scale = fp8 ? cfg.hidden / kQuantBlock : 0;
+  const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128, mx = cfg.dtype == CEP_MXFP4_E4M3;
+  const int row_bytes = cfg.hidden * (dtype_is_bytes(cfg.dtype) ? 1 : 2);
+  const int n_scale = (fp8 || mx) ? cfg.hidden / kQuantBlock : 0;       // 32-bit scale words per row
   err = launch_pdl(scatter_rows_kernel<4>, dim3(batch.n_tokens + E), dim3(kThreads), 0, s, 1, batch, k, E, row_bytes, n_scale,
                    (const int32_t*)lp.row_of_pair, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
-                   lp.pair_of_row, static_cast<uint8_t*>(xp), fp8 ? xp_scales : (float*)nullptr, cap_rows);
+                   lp.pair_of_row, static_cast<uint8_t*>(xp), (fp8 || mx) ? static_cast<uint32_t*>(xp_scales) : (uint32_t*)nullptr,
+                   mx ? 1 : 0, cap_rows);
   *launches += 4;
   return err;
 }

@@ -22,10 +22,11 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Slot {
   LayoutPtrs lp;
-  uint8_t* xp; float* xp_scales;
-  uint8_t* act; float* act_scales;
+  uint8_t* xp; void* xp_scales;
+  uint8_t* act; void* act_scales;
   uint8_t* y;
   GemmTensorMap tm_a1, tm_a2;
+  GemmTensorMap tm_sfa1, tm_sfa2;               // microscaling: scale atoms of the two activation operands
 };
 
 struct Invocation {
@@ -65,7 +66,8 @@ struct Layout {                                   // byte offsets inside the wor
 int validate(const cep_config* c, const char** why) {
   *why = nullptr;
   if (!c) { *why = "config is NULL"; return CEP_ERR_ARG; }
-  if (c->dtype != CEP_BF16 && c->dtype != CEP_FP8_E4M3_BLOCK128) { *why = "unknown dtype"; return CEP_ERR_ARG; }
+  if (c->dtype != CEP_BF16 && c->dtype != CEP_FP8_E4M3_BLOCK128 && c->dtype != CEP_MXFP4_E4M3) {
+    *why = "unknown dtype"; return CEP_ERR_ARG; }
   if (c->hidden <= 0 || c->inter <= 0 || c->hidden % 128 || c->inter % 128) {
     *why = "hidden and inter must be positive multiples of 128"; return CEP_ERR_ARG; }
   if (c->n_experts_local <= 0 || c->n_experts_local > 1024 || c->n_experts_global < c->n_experts_local) {
@@ -82,7 +84,7 @@ int validate(const cep_config* c, const char** why) {
 
 Layout make_layout(const cep_config& c) {
   Layout L{};
-  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+  const bool fp8 = dtype_is_bytes(c.dtype);       // one-byte codes + 4 bytes of scales per 128 elements
   const size_t elt = fp8 ? 1 : 2;
   const long long max_pairs = (long long)c.max_tokens * c.top_k;
   const long long pad_groups = c.n_experts_local < max_pairs ? c.n_experts_local : max_pairs;
@@ -123,13 +125,14 @@ Layout make_layout(const cep_config& c) {
 struct PackedLayout { size_t w13, w2, s13, s2, total; };
 PackedLayout make_packed_layout(const cep_config& c) {
   PackedLayout P{};
-  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128, mx = c.dtype == CEP_MXFP4_E4M3;
   const size_t elt = fp8 ? 1 : 2, E = c.n_experts_local, H = c.hidden, I = c.inter;
   size_t o = 0;
-  P.w13 = o; o = align_up(o + E * 2 * I * H * elt, 1024);
-  P.w2 = o; o = align_up(o + E * H * I * elt, 1024);
-  P.s13 = o; o = align_up(o + (fp8 ? E * (2 * I / kQuantBlock) * (H / kQuantBlock) * 4 : 0), 1024);
-  P.s2 = o; o = align_up(o + (fp8 ? E * (H / kQuantBlock) * (I / kQuantBlock) * 4 : 0), 1024);
+  // microscaling: two e2m1 codes per byte, one scale byte per 32 elements
+  P.w13 = o; o = align_up(o + (mx ? E * 2 * I * H / 2 : E * 2 * I * H * elt), 1024);
+  P.w2 = o; o = align_up(o + (mx ? E * H * I / 2 : E * H * I * elt), 1024);
+  P.s13 = o; o = align_up(o + (mx ? E * 2 * I * H / kMxBlock : fp8 ? E * (2 * I / kQuantBlock) * (H / kQuantBlock) * 4 : 0), 1024);
+  P.s2 = o; o = align_up(o + (mx ? E * H * I / kMxBlock : fp8 ? E * (H / kQuantBlock) * (I / kQuantBlock) * 4 : 0), 1024);
   P.total = o;
   return P;
 }
@@ -150,8 +153,9 @@ struct cep_plan {
   cudaEvent_t begin_evt, readback_evt, weights_evt;
   bool have_weights, layer_open, flushed, readback_pending, ever_closed;
   uint8_t* w13p; uint8_t* w2p;
-  float* s13p; float* s2p;                      // fp8: packed weight scales
+  void* s13p; void* s2p;                        // fp8, mxfp4: packed weight scales
   GemmTensorMap tm_b1, tm_b2;
+  GemmTensorMap tm_sfb1, tm_sfb2;               // mxfp4: scale atoms of the two weight operands
   // current layer call
   void* out; const void* addend; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
   std::vector<char> chunk_seen;
@@ -204,24 +208,34 @@ int launch_invocation(cep_plan* p) {
     CUDA_TRY(p, launch_layout(batch, c, sl.lp, sl.xp, sl.xp_scales, p->L.cap_rows, n_seg, st, prof ? iv.mark[3] : nullptr,
                               &p->launches));
     if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[0], st));
-    const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
+    const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128, mx = c.dtype == CEP_MXFP4_E4M3;
     const long long groups = c.n_experts_local < n_pairs ? c.n_experts_local : n_pairs;
     const long long m_tiles_bound = (n_pairs + (kRowAlign - 1) * groups + kRowAlign - 1) / kRowAlign;
-    GemmProblem g1{c.hidden, 2 * c.inter, c.n_experts_local, 1, c.inter, p->L.cap_rows, fp8};
-    GemmProblem g2{c.inter, c.hidden, c.n_experts_local, 0, c.hidden, p->L.cap_rows, fp8};
+    GemmProblem g1{c.hidden, 2 * c.inter, c.n_experts_local, 1, c.inter, p->L.cap_rows, fp8 || mx};
+    GemmProblem g2{c.inter, c.hidden, c.n_experts_local, 0, c.hidden, p->L.cap_rows, fp8 || mx};
     if (c.gemm_impl == CEP_GEMM_SIMT) {
       CUDA_TRY(p, launch_gemm_simt(g1, sl.xp, p->w13p, sl.act, sl.lp, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
       CUDA_TRY(p, launch_gemm_simt(g2, sl.act, p->w2p, sl.y, sl.lp, st, &p->launches));
+    } else if (mx) {
+      const int bn = gemm_tile_cols();
+      const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
+      const long long t1 = pair_bound * (g1.N / bn), t2 = pair_bound * (g2.N / bn);
+      CUDA_TRY(p, launch_gemm_mx(g1, sl.tm_a1, p->tm_b1, sl.tm_sfa1, p->tm_sfb1, sl.act, sl.act_scales, sl.lp,
+                                 (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
+      if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
+      CUDA_TRY(p, launch_gemm_mx(g2, sl.tm_a2, p->tm_b2, sl.tm_sfa2, p->tm_sfb2, sl.y, nullptr, sl.lp,
+                                 (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
     } else if (fp8) {
       const int pair = c.gemm_impl == CEP_GEMM_TCGEN05 ? 1 : 0;
       const int bn = gemm_tile_cols();
       const long long m_bound = pair ? (m_tiles_bound + groups + 1) / 2 : m_tiles_bound;
       const long long t1 = m_bound * ((g1.N + bn - 1) / bn), t2 = m_bound * ((g2.N + bn - 1) / bn);
-      CUDA_TRY(p, launch_gemm_fp8(g1, pair, sl.tm_a1, p->tm_b1, sl.xp_scales, p->s13p, sl.act, sl.act_scales, sl.lp,
+      CUDA_TRY(p, launch_gemm_fp8(g1, pair, sl.tm_a1, p->tm_b1, (const float*)sl.xp_scales, (const float*)p->s13p, sl.act,
+                                  (float*)sl.act_scales, sl.lp,
                                   (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
-      CUDA_TRY(p, launch_gemm_fp8(g2, pair, sl.tm_a2, p->tm_b2, sl.act_scales, p->s2p, sl.y, nullptr, sl.lp,
+      CUDA_TRY(p, launch_gemm_fp8(g2, pair, sl.tm_a2, p->tm_b2, (const float*)sl.act_scales, (const float*)p->s2p, sl.y, nullptr, sl.lp,
                                   (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
     } else if (c.gemm_impl == CEP_GEMM_TCGEN05) {
       const int bn = gemm_tile_cols();
@@ -287,6 +301,11 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
       return fail(nullptr, CEP_ERR_UNSUPPORTED, "block-scaled fp8 runs on the tensor-core kernels only");
     if (cfg->hidden % 256) return fail(nullptr, CEP_ERR_ARG, "fp8 needs hidden to be a multiple of 256");
   }
+  if (cfg->dtype == CEP_MXFP4_E4M3) {
+    if (cfg->gemm_impl != CEP_GEMM_TCGEN05)
+      return fail(nullptr, CEP_ERR_UNSUPPORTED, "microscaling operands run on the CTA-pair tensor-core kernel only");
+    if (cfg->hidden % 256) return fail(nullptr, CEP_ERR_ARG, "mxfp4 needs hidden to be a multiple of 256");
+  }
   Layout L = make_layout(*cfg);
   if (workspace_bytes < L.total) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return fail(nullptr, CEP_ERR_WORKSPACE, "workspace must be 256-byte aligned");
@@ -320,8 +339,8 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     if (cfg->profile_kernels)
       for (int m = 0; m < 4; ++m) { PLAN_TRY(cudaEventCreate(&e)); p->inv_mark.push_back(e); }
   }
-  const bool fp8 = cfg->dtype == CEP_FP8_E4M3_BLOCK128;
-  const int elt = fp8 ? 1 : 2;
+  const bool mx = cfg->dtype == CEP_MXFP4_E4M3;
+  const int elt = dtype_is_bytes(cfg->dtype) ? 1 : 2;
   for (int s = 0; s < cfg->n_streams; ++s) {
     uint8_t* b = p->ws + L.slot0 + L.slot_bytes * s;
     Slot sl{};
@@ -334,12 +353,16 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     sl.lp.pair_of_row = reinterpret_cast<int32_t*>(b + L.pair_of_row);
     sl.lp.status = reinterpret_cast<int32_t*>(p->ws + L.status);
     sl.lp.sched = reinterpret_cast<int32_t*>(b + L.sched);
-    sl.xp = b + L.xp; sl.xp_scales = reinterpret_cast<float*>(b + L.xp_scales);
-    sl.act = b + L.act; sl.act_scales = reinterpret_cast<float*>(b + L.act_scales);
+    sl.xp = b + L.xp; sl.xp_scales = b + L.xp_scales;
+    sl.act = b + L.act; sl.act_scales = b + L.act_scales;
     sl.y = b + L.y;
     if (cfg->gemm_impl != CEP_GEMM_SIMT) {
       int r1 = make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
       int r2 = make_operand_map(&sl.tm_a2, sl.act, elt, cfg->inter, L.cap_rows, 0, gemm_tile_rows());
+      if (mx && !r1 && !r2) {
+        r1 = make_mx_sf_map(&sl.tm_sfa1, sl.xp_scales, (long long)(L.cap_rows / kRowAlign) * (cfg->hidden / 128), kSfAtomBytes);
+        r2 = make_mx_sf_map(&sl.tm_sfa2, sl.act_scales, (long long)(L.cap_rows / kRowAlign) * (cfg->inter / 128), kSfAtomBytes);
+      }
       if (r1 || r2) {
         fail(nullptr, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the activation operands failed (%d, %d)", r1, r2);
         moe_plan_destroy(p);
@@ -358,24 +381,39 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   return CEP_OK;
 }
 
-int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const void* w_down, const float* s_gate,
-                     const float* s_up, const float* s_down, void* packed, size_t packed_bytes, void* stream) {
+int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const void* w_down, const void* s_gate,
+                     const void* s_up, const void* s_down, void* packed, size_t packed_bytes, void* stream) {
   if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
   if (!w_gate || !w_up || !w_down || !packed) return fail(p, CEP_ERR_ARG, "a weight pointer is NULL");
   if (p->layer_open) return fail(p, CEP_ERR_STATE, "weights cannot change while a layer call is open");
   const cep_config& c = p->cfg;
-  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128;
-  if (fp8 && (!s_gate || !s_up || !s_down)) return fail(p, CEP_ERR_ARG, "fp8 weights need their scale tensors");
+  const bool fp8 = c.dtype == CEP_FP8_E4M3_BLOCK128, mx = c.dtype == CEP_MXFP4_E4M3;
+  if ((fp8 || mx) && (!s_gate || !s_up || !s_down)) return fail(p, CEP_ERR_ARG, "quantised weights need their scale tensors");
   PackedLayout P = make_packed_layout(c);
   if (packed_bytes < P.total) return fail(p, CEP_ERR_WORKSPACE, "packed buffer has %zu bytes, %zu needed", packed_bytes, P.total);
   if (reinterpret_cast<uintptr_t>(packed) % 256) return fail(p, CEP_ERR_WORKSPACE, "packed buffer must be 256-byte aligned");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   p->w13p = static_cast<uint8_t*>(packed) + P.w13;
   p->w2p = static_cast<uint8_t*>(packed) + P.w2;
-  p->s13p = reinterpret_cast<float*>(static_cast<uint8_t*>(packed) + P.s13);
-  p->s2p = reinterpret_cast<float*>(static_cast<uint8_t*>(packed) + P.s2);
+  p->s13p = static_cast<uint8_t*>(packed) + P.s13;
+  p->s2p = static_cast<uint8_t*>(packed) + P.s2;
+  if (mx) {
+    CUDA_TRY(p, launch_prepack_mx(c, w_gate, w_up, w_down, s_gate, s_up, s_down, p->w13p, p->w2p, p->s13p, p->s2p, st,
+                                  &p->launches));
+    CUDA_TRY(p, cudaEventRecord(p->weights_evt, st));
+    const int box = gemm_tile_cols() / 2, E = c.n_experts_local;
+    int r1 = make_mx_weight_map(&p->tm_b1, p->w13p, c.hidden, 2 * c.inter, E, box);
+    int r2 = make_mx_weight_map(&p->tm_b2, p->w2p, c.inter, c.hidden, E, box);
+    int r3 = make_mx_sf_map(&p->tm_sfb1, p->s13p, (long long)E * (2 * c.inter / 256) * (c.hidden / 128), 2 * kSfAtomBytes);
+    int r4 = make_mx_sf_map(&p->tm_sfb2, p->s2p, (long long)E * (c.hidden / 256) * (c.inter / 128), 2 * kSfAtomBytes);
+    if (r1 || r2 || r3 || r4)
+      return fail(p, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the weight operands failed (%d, %d, %d, %d)", r1, r2, r3, r4);
+    p->have_weights = true;
+    return CEP_OK;
+  }
   CUDA_TRY(p, launch_prepack(c, w_gate, w_up, w_down, p->w13p, p->w2p, st, &p->launches));
-  if (fp8) CUDA_TRY(p, launch_pack_scales(c, s_gate, s_up, s_down, p->s13p, p->s2p, st, &p->launches));
+  if (fp8) CUDA_TRY(p, launch_pack_scales(c, (const float*)s_gate, (const float*)s_up, (const float*)s_down, (float*)p->s13p,
+                                          (float*)p->s2p, st, &p->launches));
   CUDA_TRY(p, cudaEventRecord(p->weights_evt, st));
   if (c.gemm_impl != CEP_GEMM_SIMT) {
     const int elt = fp8 ? 1 : 2;
@@ -410,7 +448,7 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
 }
 
 int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_t n_tokens, const void* tokens,
-                     const float* token_scales, const int32_t* topk_ids, const float* topk_weights,
+                     const void* token_scales, const int32_t* topk_ids, const float* topk_weights,
                      int64_t n_local_pairs, void* stream) {
   if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
   if (!p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_submit_chunk before ffn_begin");
@@ -421,8 +459,9 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   if ((long long)token_offset + n_tokens > p->n_tokens_total) return fail(p, CEP_ERR_CAPACITY, "chunk %d covers tokens beyond n_tokens_total", chunk_id);
   if (n_tokens > 0 && (!tokens || !topk_ids || !topk_weights)) return fail(p, CEP_ERR_ARG, "a chunk pointer is NULL");
   if (reinterpret_cast<uintptr_t>(tokens) % 16) return fail(p, CEP_ERR_ARG, "chunk tokens must be 16-byte aligned");
-  const bool fp8 = p->cfg.dtype == CEP_FP8_E4M3_BLOCK128;
-  if (fp8 && n_tokens > 0 && !token_scales) return fail(p, CEP_ERR_ARG, "fp8 chunk without token_scales");
+  const bool fp8 = dtype_is_bytes(p->cfg.dtype);
+  if (fp8 && n_tokens > 0 && !token_scales) return fail(p, CEP_ERR_ARG, "quantised chunk without token_scales");
+  if (fp8 && reinterpret_cast<uintptr_t>(token_scales) % 4) return fail(p, CEP_ERR_ARG, "token_scales must be 4-byte aligned");
   const int64_t bound = (int64_t)n_tokens * p->cfg.top_k;
   if (n_local_pairs > bound) return fail(p, CEP_ERR_ARG, "n_local_pairs exceeds n_tokens*top_k");
   const int64_t pairs = n_local_pairs < 0 ? bound : n_local_pairs;

@@ -24,7 +24,7 @@ def sweep(name="straggler", taus=(0.0, 0.5), streams=(1, 2, 4), warm=3, reps=10,
     pairs = [int((c[3] < cfg.E_local).sum().item()) for c in chunks]
     out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device=device)
     rstreams = [torch.cuda.Stream() for _ in chunks]
-    dt = cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16
+    dt = cep.DTYPE_OF[cfg.dtype]
 
     def measure(mode, theta, S, arrival):
         L = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt, mode=mode,

@@ -20,7 +20,7 @@ def chunks_of(inp):
 
 def make_layer(cfg, mode=cep.CEP_MODE_SYNC, theta=0, n_streams=2, gemm_impl=cep.CEP_GEMM_TCGEN05, max_chunks=None,
                debug_checks=0):
-    dt = cep.CEP_FP8_E4M3_BLOCK128 if cfg.dtype == "fp8" else cep.CEP_BF16
+    dt = cep.DTYPE_OF[cfg.dtype]
     return cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, max_chunks or max(cfg.n_chunks, 1),
                         dtype=dt, mode=mode, n_streams=n_streams, threshold_pairs=theta, gemm_impl=gemm_impl,
                         debug_checks=debug_checks)
