@@ -94,7 +94,9 @@ def workload_numbers(cfg, n_pairs):
     """Algorithmic work of one step: 6*H*I FLOP per kept (token, expert) pair; bytes per kernel as the method
     itself must move them (each row read/written once, each touched expert's weights read once)."""
     H, I, T, E = cfg.H, cfg.I, cfg.T, cfg.E_local
-    s = 2 if cfg.dtype == "bf16" else 1 + 4.0 / 128      # bytes per element (fp8: code + its share of a 1x128 scale)
+    s = 2 if cfg.dtype == "bf16" else 1 + 4.0 / 128      # bytes per element (fp8: code + its share of a 1x128 scale;
+    #                                                      mxfp4 activations: e4m3 code + 1/32 of a scale byte: the same)
+    sw = 0.5 + 1.0 / 32 if cfg.dtype == "mxfp4" else s   # bytes per weight element (mxfp4: a nibble + 1/32 scale byte)
     return {
         "pairs": n_pairs,
         "flops": 6.0 * H * I * n_pairs,
@@ -102,8 +104,8 @@ def workload_numbers(cfg, n_pairs):
         "gemm2_flops": 2.0 * H * I * n_pairs,
         "layout_bytes": (T + n_pairs) * H * s + T * cfg.k * 4.0,
         "combine_bytes": (n_pairs + T) * H * 2.0 + n_pairs * 4.0,
-        "gemm1_bytes": n_pairs * H * s + 2.0 * H * I * s * E + n_pairs * I * s,
-        "gemm2_bytes": n_pairs * I * s + 1.0 * H * I * s * E + n_pairs * H * 2,
+        "gemm1_bytes": n_pairs * H * s + 2.0 * H * I * sw * E + n_pairs * I * s,
+        "gemm2_bytes": n_pairs * I * s + 1.0 * H * I * sw * E + n_pairs * H * 2,
     }
 
 
@@ -408,13 +410,14 @@ def main():
     sustained = capped or (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
     peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     nominal_tf = NOMINAL_BF16_TFLOPS
-    if cfg.dtype == "fp8":          # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2)
+    if cfg.dtype in ("fp8", "mxfp4"):   # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2);
+        #                                 the mxf8f6f4 MMA kind (e4m3 x e2m1) runs at the fp8 rate
         peak_tf, nominal_tf = 2.0 * peak_tf, 2.0 * NOMINAL_BF16_TFLOPS
     roofline = {"bound": "tensor", "kernel": "grouped GEMM1 (gate/up + SiLU*up%s), CTA-pair tcgen05" %
-                          (" + e4m3 re-quantisation" if cfg.dtype == "fp8" else ""),
+                          (" + e4m3 re-quantisation" if cfg.dtype != "bf16" else ""),
                 "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
                 "peak_kind": ("sustained" if sustained else "burst") + " bf16 cuBLAS" +
-                             (" x2 (nominal fp8:bf16 ratio)" if cfg.dtype == "fp8" else "") + ", of " + peaks["source"],
+                             (" x2 (nominal fp8:bf16 ratio)" if cfg.dtype != "bf16" else "") + ", of " + peaks["source"],
                 "frac_of_nominal": g1_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                 "duration_ms": g1_ms, "traffic": None}
     roofline["traffic"] = GEMM1_DRAM_TRAFFIC.get(cfg.name)
@@ -431,12 +434,12 @@ def main():
     }
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "fp8_e4m3", "data": "synthetic",
+            "vs_baseline": None, "dtype": {"bf16": "bf16", "fp8": "fp8_e4m3", "mxfp4": "e4m3 x e2m1 (ue8m0 1x32 scales)"}[cfg.dtype], "data": "synthetic",
             "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E_local": cfg.E_local,
                        "E_global": cfg.E_global, "top_k": cfg.k, "local_pairs": n_pairs, "chunks": list(cfg.chunks),
                        "mode": "sync (one invocation, all chunks present)", "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (weights %.2f GB re-read every step)" %
-                             (3.0 * cfg.H * cfg.I * (2 if cfg.dtype == "bf16" else 1) * cfg.E_local / 1e9)},
+                             (3.0 * cfg.H * cfg.I * {"bf16": 2, "fp8": 1, "mxfp4": 0.5}[cfg.dtype] * cfg.E_local / 1e9)},
             "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal": ffn_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                            "frac_of_measured": ffn_tflops / peak_tf, "flops_per_step": work["flops"]},
             "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e, "streamffn": stream_report,

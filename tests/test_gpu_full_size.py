@@ -40,13 +40,13 @@ def sample_tokens(inp, n_random=40, seed=0):
     return np.unique(np.array(sel, dtype=np.int64))
 
 
-@pytest.mark.parametrize("name", ["ep_shard", "ep_shard_strided"])
+@pytest.mark.parametrize("name", ["ep_shard", "ep_shard_strided", "mxfp4_shard"])
 def test_ep_shard_full_size(name):
     cfg = wl.CONFIGS[name]
     inp = wl.make_inputs(cfg, device="cuda", keep_logits=False)
     host = host_view(inp)
     layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, debug_checks=1)
-    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     out, n_inv = run_layer(inp, layer, local_pairs=True)
     assert n_inv == 1
     assert cep.cep_debug_check_guards(layer.plan) == 0
@@ -68,7 +68,7 @@ def test_ep_shard_full_size(name):
     assert (out[~none_local].float().abs().sum(dim=1) > 0).all()
     # chunked asynchronous execution gives the same bits as the one synchronous launch
     stream = make_layer(cfg, mode=cep.CEP_MODE_STREAMFFN, theta=max(1, host.n_local_pairs() // 3), n_streams=2)
-    stream.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+    stream.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     out2, n_inv2 = run_layer(inp, stream, order=wl.submission_order(host.arrival), local_pairs=True)
     assert n_inv2 > 1
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))

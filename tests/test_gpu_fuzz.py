@@ -15,7 +15,8 @@ pytestmark = pytest.mark.gpu
 
 def random_config(seed):
     r = np.random.default_rng(1000 + seed)
-    fp8 = seed % 4 == 3
+    mx = seed >= 24                       # the last eight seeds draw microscaling configurations
+    fp8 = seed % 4 == 3 or mx             # both quantised formats need hidden to be a multiple of 256
     H = int(r.choice([256, 512, 768, 1024])) if fp8 else int(r.choice([128, 256, 384, 640, 1024]))
     I = int(r.choice([128, 256, 384, 512]))
     E_global = int(r.choice([1, 2, 5, 8, 24, 64, 130]))
@@ -26,7 +27,7 @@ def random_config(seed):
     cuts = np.sort(r.choice(np.arange(T + 1), size=n_chunks - 1, replace=True)) if n_chunks > 1 else np.array([], int)
     sizes = np.diff(np.concatenate([[0], cuts, [T]])).astype(int).tolist()
     cfg = wl.MoEConfig("fuzz%d" % seed, seed % 5, T=T, H=H, I=I, E_global=E_global, E_local=E_local, k=k,
-                       chunks=tuple(sizes), dtype="fp8" if fp8 else "bf16", zipf_s=float(r.choice([0.0, 1.1])))
+                       chunks=tuple(sizes), dtype="mxfp4" if mx else ("fp8" if fp8 else "bf16"), zipf_s=float(r.choice([0.0, 1.1])))
     mode = int(r.choice([cep.CEP_MODE_SYNC, cep.CEP_MODE_ASYNC, cep.CEP_MODE_STREAMFFN]))
     theta = int(r.integers(0, max(2, T * k)))
     S = int(r.integers(1, 4))
@@ -34,7 +35,7 @@ def random_config(seed):
     return cfg, mode, theta, S, order
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(32))
 def test_random_configuration(seed):
     cfg, mode, theta, S, order = random_config(seed)
     host = wl.make_inputs(cfg)
