@@ -297,13 +297,6 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     _Pragma("unroll") for (int i = 0; i < 16; ++i)                                                  \
         fma_f32x2(acc2[(BASE) + i], pack_f32x2((V)[2 * i], (V)[2 * i + 1]), s2_);                  \
   }
-#ifdef CEP_EXP_NO_TMEM_LD
-#define tc_ld32(addr, v) { (v)[0] = (addr); (v)[1] = 0; }
-#endif
-#ifdef CEP_EXP_NO_FMA
-#undef CEP_FMA_CHUNK
-#define CEP_FMA_CHUNK(V, BASE, S) { acc2[(BASE)] += (V)[0] + (V)[1] + __float_as_uint(S); }
-#endif
       uint32_t va[32], vb[32];
       {
         const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);

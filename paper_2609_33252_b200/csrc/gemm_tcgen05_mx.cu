@@ -20,6 +20,12 @@
 //   GEMM2  bf16
 // Roles (384 threads): warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader CTA), warp 2 tile scheduler
 // (leader CTA), warps 4-11 epilogue.  Tiles come from a global counter.  All waits are bounded.
+//
+// Where the time goes (device-timer trace and profiler counters on the 7168x2048 shapes): a K=128 slab costs
+// about 470 cycles of MMA, 115 cycles for its three scale copies (they run in the same in-order pipe as the MMAs;
+// issuing them a slab ahead or leaving them out confirms it: 2640 TFLOP/s without copies, the same as an unscaled
+// kind::f8f6f4 loop), and the rest is the issue thread's barrier round trip per group of slabs.  The tile-end
+// bubble is small: the finished accumulator is in registers 160 cycles after the epilogue warps see it.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -38,7 +44,13 @@ constexpr int B_STAGE = (BN / 2) * BKE;                // this CTA's half of the
 constexpr int B_TX = (BN / 2) * BKE / 2;               // bytes the TMA engine counts for it (packed codes)
 constexpr int SFA_STAGE = kSfAtomBytes;                // 128 rows x 4 scale blocks
 constexpr int SFB_STAGE = 2 * kSfAtomBytes;            // 256 weight rows x 4 scale blocks
-constexpr int kStages = 6;
+constexpr int kStages = 6;                             // K=128 slabs of operands in shared memory
+// Slabs are handed between producer and MMA warp two at a time: one barrier round trip (wait, fence, commit) per
+// eight MMAs instead of four.  Measured on the 7168x2048 expert shapes: GEMM1 2260 -> 2390 TFLOP/s, GEMM2 2206 ->
+// 2280; three at a time helps the long-K GEMM1 a little more but leaves the K=2048 GEMM2 only two rounds deep.
+constexpr int kGroup = 2;
+constexpr int kRounds = kStages / kGroup;
+static_assert(kStages % kGroup == 0, "slabs per round");
 constexpr int kThreads = 384;
 constexpr int kEpiWarp0 = 4, kEpiWarps = 8;
 constexpr int kTmemCols = 512;
@@ -51,7 +63,7 @@ constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE + SFA_STAGE + SFB_STAGE)
 constexpr uint32_t kStageTx = 2u * (A_STAGE + B_TX + SFA_STAGE + SFB_STAGE);   // both CTAs' bytes, counted at the leader
 
 struct __align__(8) Bars {
-  uint64_t full[kStages], empty[kStages];
+  uint64_t full[kRounds], empty[kRounds];
   uint64_t acc_full, acc_empty;
   uint64_t sched_full[kRing], sched_empty[kRing];
   int32_t sched_tile[kRing];
@@ -148,7 +160,7 @@ grouped_gemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   volatile int* abort_flag = &bars->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
+    for (int s = 0; s < kRounds; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
     mbar_init(smem_u32(&bars->acc_full), 1);
     mbar_init(smem_u32(&bars->acc_empty), 2 * kEpiWarps);
     for (int s = 0; s < kRing; ++s) {
@@ -196,15 +208,19 @@ grouped_gemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
         const int n0 = tc.n_block * BN + (int)rank * (BN / 2);
         const int sfa_atom0 = (row0 >> 7) * num_kb;                                   // atoms are [row block][k128]
         const int sfb_atom0 = (tc.expert * n_blocks_n + tc.n_block) * num_kb;         // [expert][n block of 256][k128]
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb0 = 0; kb0 < num_kb; kb0 += kGroup) {        // `stage` counts rounds of kGroup slabs here
+          const int n_sub = num_kb - kb0 < kGroup ? num_kb - kb0 : kGroup;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
           const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);
-          if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), kStageTx);
-          tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * BKE, row0, full);
-          tma_load_3d_pair(smem_u32(smem_b + stage * B_STAGE), &tm_b, kb * BKE, n0, tc.expert, full);
-          tma_load_2d_pair(smem_u32(smem_sfa + stage * SFA_STAGE), &tm_sfa, 0, sfa_atom0 + kb, full);
-          tma_load_2d_pair(smem_u32(smem_sfb + stage * SFB_STAGE), &tm_sfb, 0, sfb_atom0 + kb, full);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), (uint32_t)n_sub * kStageTx);
+          for (int sub = 0; sub < n_sub; ++sub) {
+            const int slab = stage * kGroup + sub, kb = kb0 + sub;
+            tma_load_2d_pair(smem_u32(smem_a + slab * A_STAGE), &tm_a, kb * BKE, row0, full);
+            tma_load_3d_pair(smem_u32(smem_b + slab * B_STAGE), &tm_b, kb * BKE, n0, tc.expert, full);
+            tma_load_2d_pair(smem_u32(smem_sfa + slab * SFA_STAGE), &tm_sfa, 0, sfa_atom0 + kb, full);
+            tma_load_2d_pair(smem_u32(smem_sfb + slab * SFB_STAGE), &tm_sfb, 0, sfb_atom0 + kb, full);
+          }
+          if (++stage == kRounds) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1 && lane == 0 && !is_peer) {
@@ -220,23 +236,27 @@ grouped_gemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
         if (tile < 0) break;
         if (!mbar_wait(smem_u32(&bars->acc_empty), acc_phase ^ 1u, abort_flag, status)) break;
         tc_fence_after();
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb0 = 0; kb0 < num_kb; kb0 += kGroup) {
+          const int n_sub = num_kb - kb0 < kGroup ? num_kb - kb0 : kGroup;
           if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sfa_t = tmem_base + (uint32_t)(kSfCol0 + sf_slot * kSfSlotCols);
-          const uint32_t sfb_t = sfa_t + 4u;
-          tc_cp_sf_pair(sfa_t, make_sf_desc(smem_u32(smem_sfa + stage * SFA_STAGE)));
-          tc_cp_sf_pair(sfb_t, make_sf_desc(smem_u32(smem_sfb + stage * SFB_STAGE)));
-          tc_cp_sf_pair(sfb_t + 4u, make_sf_desc(smem_u32(smem_sfb + stage * SFB_STAGE + kSfAtomBytes)));
-          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE));
-          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * B_STAGE));
+          for (int sub = 0; sub < n_sub; ++sub) {
+            const int slab = stage * kGroup + sub;
+            const uint32_t sfa_t = tmem_base + (uint32_t)(kSfCol0 + sf_slot * kSfSlotCols);
+            const uint32_t sfb_t = sfa_t + 4u;
+            tc_cp_sf_pair(sfa_t, make_sf_desc(smem_u32(smem_sfa + slab * SFA_STAGE)));
+            tc_cp_sf_pair(sfb_t, make_sf_desc(smem_u32(smem_sfb + slab * SFB_STAGE)));
+            tc_cp_sf_pair(sfb_t + 4u, make_sf_desc(smem_u32(smem_sfb + slab * SFB_STAGE + kSfAtomBytes)));
+            const uint64_t adesc = make_smem_desc(smem_u32(smem_a + slab * A_STAGE));
+            const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + slab * B_STAGE));
 #pragma unroll
-          for (int k4 = 0; k4 < BKE / 32; ++k4)          // 32 elements of K per MMA = one scale block
-            tc_mma_mx_pair(tmem_base, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), make_idesc_mx(2 * BM, BN, k4),
-                           sfa_t, sfb_t, (kb | k4) != 0 ? 1u : 0u);
+            for (int k4 = 0; k4 < BKE / 32; ++k4)        // 32 elements of K per MMA = one scale block
+              tc_mma_mx_pair(tmem_base, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), make_idesc_mx(2 * BM, BN, k4),
+                             sfa_t, sfb_t, (kb0 | sub | k4) != 0 ? 1u : 0u);
+            if (++sf_slot == kSfSlots) sf_slot = 0;
+          }
           tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          if (++sf_slot == kSfSlots) sf_slot = 0;
+          if (++stage == kRounds) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         tc_commit_pair_both(smem_u32(&bars->acc_full), 3);
