@@ -27,9 +27,11 @@ METRIC = "MoE-layer prefill tokens/s (streamFFN routed-expert path: permute + gr
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM1 launch, from the ncu captures summarised in
-# profiles/grouped_gemm_bf16_pair_ep_shard.md and profiles/grouped_gemm_fp8_pair_fp8_shard_small.md
+# profiles/grouped_gemm_bf16_pair_ep_shard.md, profiles/grouped_gemm_fp8_pair_fp8_shard_small.md and
+# profiles/grouped_gemm_mx_pair_mxfp4_shard.md
 GEMM1_DRAM_TRAFFIC = {"ep_shard": 5.64e9 + 0.51e9, "straggler": 5.64e9 + 0.51e9,
-                      "ep_shard_small": 1.02e9 + 0.041e9, "fp8_shard_small": 0.462e9 + 0.034e9}
+                      "ep_shard_small": 1.02e9 + 0.041e9, "fp8_shard_small": 0.462e9 + 0.034e9,
+                      "mxfp4_shard": 1.427e9 + 0.260e9, "mxfp4_shard_small": 0.204e9 + 0.019e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
