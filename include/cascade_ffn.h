@@ -254,6 +254,52 @@ CEP_API int ffn_query(cep_plan* plan, int32_t inv, cep_invocation_info* info);
 CEP_API int ffn_debug_export(cep_plan* plan, int32_t inv, int32_t* counts, int32_t* offsets,
                      int32_t* padded_offsets, int32_t* row_of_pair, int32_t* pair_of_row);
 
+/*
+ * Use only the first `n` (1..n_streams) compute streams / scratch slots for the following layer calls
+ * (round-robin over n instead of n_streams).  Between layer calls only.  A plan starts with all of them.
+ */
+CEP_API int ffn_set_active_streams(cep_plan* plan, int32_t n);
+
+/* One point of the FFN-throughput profile (the quantity plotted against expert-token count in Section 3.2,
+ * "Launch threshold"): every local expert gets the same number of rows. */
+typedef struct {
+  int32_t rows_per_expert;
+  int32_t n_tokens;            /* tokens of the synthetic batch                                   */
+  int64_t expert_tokens;       /* N: local (token, expert) pairs of the batch                     */
+  float ffn_ms;                /* F(N): median device time of the two expert GEMMs                */
+  float layer_ms;              /* median device time of the whole invocation                      */
+  float tflops;                /* 6*H*I*N / F(N)                                                  */
+  float eta;                   /* tflops / peak of the profile: F(N) = N / (eta(N) * P_peak)      */
+} cep_profile_point;
+
+typedef struct {
+  float rho;                   /* throughput target given                                         */
+  float peak_tflops;           /* best point of the profile (P_peak)                              */
+  int64_t theta_pairs;         /* smallest profiled N with eta(N) >= rho                          */
+  int32_t theta_rows_per_expert;
+  int32_t best_streams;        /* fewest active streams within 2 % of the fastest probe; 0 if not probed */
+  int32_t probe_invocations;   /* invocations of theta_pairs each in the stream probe             */
+  float stream_ms[16];         /* median completion time of the probe with s+1 active streams; < 0: not run */
+} cep_calibration;
+
+/*
+ * Launch-threshold calibration (Section 3.2: theta is "the smallest profiled count that reaches at least rho of
+ * the observed peak FFN throughput"; Section 4.2 models FFN latency from the same profile).  Runs the plan's OWN
+ * kernels, with the weights it holds, on synthetic routing that gives every local expert rows_per_expert[i] rows
+ * (ascending), `reps` timed layer calls per point after two warm-ups, and then probes how many compute streams a
+ * chain of theta-sized invocations wants.  Blocks the host until done; not part of the hot path.  Needs a plan
+ * made with profile_kernels != 0, loaded weights, no open layer call.  Caller-provided [device] scratch, for
+ * T_max = max(rows_per_expert) * n_experts_local / min(top_k, n_experts_local) tokens (T_max <= max_tokens):
+ *   tokens        [T_max, H] in the plan's activation format, any finite values (they are only timed)
+ *   token_scales  as for ffn_submit_chunk, or NULL for bf16
+ *   ids, weights  [T_max, top_k] int32 / fp32, overwritten with the synthetic routing
+ *   out           [T_max, H] bf16, overwritten
+ * [host] out: points[n_points], *result.  The plan's mode, threshold and active streams are restored on return.
+ */
+CEP_API int cep_calibrate(cep_plan* plan, float rho, const int32_t* rows_per_expert, int32_t n_points, int32_t reps,
+                          const void* tokens, const void* token_scales, int32_t* ids, float* weights, void* out,
+                          cep_profile_point* points, cep_calibration* result);
+
 /* Total kernel launches this plan has issued (layout, GEMM, combine, prepack). */
 CEP_API int64_t cep_kernel_launches(const cep_plan* plan);
 

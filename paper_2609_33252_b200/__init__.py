@@ -10,5 +10,6 @@ from .binding import (CepConfig, CepError, InvocationInfo, MoELayer, lib, load_l
                       ffn_begin, ffn_set_addend, moe_route, ffn_submit_chunk, ffn_flush, combine, ffn_status, ffn_num_invocations, ffn_wait_invocation,
                       ffn_query, ffn_debug_export, cep_kernel_launches, moe_plan_destroy, cep_last_error,
                       cep_debug_decode_tile, cep_debug_schedule, layout_indices_noalloc, cep_debug_wait_timeout, cep_debug_check_guards,
+                      ffn_set_active_streams, cep_calibrate,
                       CEP_BF16, CEP_FP8_E4M3_BLOCK128, CEP_MXFP4_E4M3, DTYPE_OF, CEP_MODE_SYNC, CEP_MODE_ASYNC, CEP_MODE_STREAMFFN,
                       CEP_GEMM_TCGEN05, CEP_GEMM_SIMT, CEP_GEMM_TCGEN05_1CTA, STATUS_NAMES)

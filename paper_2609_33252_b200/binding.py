@@ -24,7 +24,8 @@ STATUS_NAMES = {0: "CEP_OK", -1: "CEP_ERR_ARG", -2: "CEP_ERR_STATE", -3: "CEP_ER
 EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "moe_load_weights",
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
-           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards", "ffn_wait_invocation"]
+           "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards", "ffn_wait_invocation",
+           "ffn_set_active_streams", "cep_calibrate"]
 
 
 class CepConfig(ctypes.Structure):
@@ -43,6 +44,18 @@ class InvocationInfo(ctypes.Structure):
                 ("pairs_bound", ctypes.c_int64), ("elapsed_ms", ctypes.c_float),
                 ("layout_ms", ctypes.c_float), ("gemm1_ms", ctypes.c_float), ("gemm2_ms", ctypes.c_float),
                 ("combine_ms", ctypes.c_float), ("index_ms", ctypes.c_float), ("scatter_ms", ctypes.c_float)]
+
+
+class ProfilePoint(ctypes.Structure):
+    _fields_ = [("rows_per_expert", ctypes.c_int32), ("n_tokens", ctypes.c_int32), ("expert_tokens", ctypes.c_int64),
+                ("ffn_ms", ctypes.c_float), ("layer_ms", ctypes.c_float), ("tflops", ctypes.c_float),
+                ("eta", ctypes.c_float)]
+
+
+class Calibration(ctypes.Structure):
+    _fields_ = [("rho", ctypes.c_float), ("peak_tflops", ctypes.c_float), ("theta_pairs", ctypes.c_int64),
+                ("theta_rows_per_expert", ctypes.c_int32), ("best_streams", ctypes.c_int32),
+                ("probe_invocations", ctypes.c_int32), ("stream_ms", ctypes.c_float * 16)]
 
 
 class CepError(RuntimeError):
@@ -94,6 +107,9 @@ def load_library(build_if_missing: bool = True):
         "ffn_set_addend": (ctypes.c_int, [vp, vp]),
         "cep_debug_check_guards": (ctypes.c_int, [vp, ctypes.POINTER(i32)]),
         "moe_route": (ctypes.c_int, [vp, i32, i32, i32, vp, vp, vp]),
+        "ffn_set_active_streams": (ctypes.c_int, [vp, i32]),
+        "cep_calibrate": (ctypes.c_int, [vp, ctypes.c_float, vp, i32, i32, vp, vp, vp, vp, vp,
+                                         ctypes.POINTER(ProfilePoint), ctypes.POINTER(Calibration)]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -213,6 +229,24 @@ def ffn_debug_export(plan, inv: int, n_experts_local: int, n_pairs: int):
     _check(lib().ffn_debug_export(plan, inv, None, None, None, None, p(por)), plan)
     return dict(counts=counts, offsets=offsets, padded_offsets=padded, row_of_pair=rop[:n_pairs],
                 pair_of_row=por[:int(padded[E])])
+
+
+def ffn_set_active_streams(plan, n: int):
+    _check(lib().ffn_set_active_streams(plan, n), plan)
+
+
+def cep_calibrate(plan, rho: float, rows_per_expert: Sequence[int], reps: int, tokens, token_scales, ids, weights, out):
+    """Returns (list of profile-point dicts, calibration dict); the tensors are device scratch (see the header)."""
+    n = len(rows_per_expert)
+    rows = (ctypes.c_int32 * n)(*[int(r) for r in rows_per_expert])
+    pts = (ProfilePoint * n)()
+    cal = Calibration()
+    _check(lib().cep_calibrate(plan, float(rho), ctypes.cast(rows, ctypes.c_void_p), n, reps, _dptr(tokens),
+                               _dptr(token_scales), _dptr(ids), _dptr(weights), _dptr(out), pts, ctypes.byref(cal)), plan)
+    points = [{f: getattr(p, f) for f, _ in ProfilePoint._fields_} for p in pts]
+    result = {f: getattr(cal, f) for f, _ in Calibration._fields_ if f != "stream_ms"}
+    result["stream_ms"] = [v for v in cal.stream_ms if v >= 0]
+    return points, result
 
 
 def cep_kernel_launches(plan) -> int:

@@ -78,6 +78,38 @@ def calibrate(cfg: wl.MoEConfig, rho: float = 0.90, **kw) -> Dict:
             "theta_rows_per_expert": theta // cfg.E_local, "profile": prof}
 
 
+def calibrate_in_library(cfg: wl.MoEConfig, rho: float = 0.90, rows: Sequence[int] = (64, 128, 256, 512, 1024, 2048),
+                         reps: int = 5, n_streams: int = 4, device="cuda") -> Dict:
+    """The same calibration done by the library itself (``cep_calibrate``): profile, theta(rho) and the number of
+    compute streams a chain of theta-sized invocations wants.  This wrapper only allocates the scratch tensors."""
+    import torch
+    inp = wl.make_inputs(wl.scaled(cfg, T=8, chunks=(8,)), device=device, keep_logits=False)   # weights only
+    E, k, H, I = cfg.E_local, cfg.k, cfg.H, cfg.I
+    k_loc = min(k, E)
+    T_max = max(1, max(rows) * E // k_loc)
+    layer = cep.MoELayer(H, I, cfg.E_global, E, k, T_max, 8, dtype=cep.DTYPE_OF[cfg.dtype], mode=cep.CEP_MODE_SYNC,
+                         n_streams=n_streams, profile_kernels=1)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+    x32 = torch.randn((T_max, H), generator=torch.Generator(device=device).manual_seed(wl.SEED_BASE + 99), device=device)
+    if cfg.dtype == "fp8":
+        x, xs = wl.quantize_rows_1x128(x32)
+    elif cfg.dtype == "mxfp4":
+        x, xs = wl.quantize_mx(x32, "e4m3", 1)
+    else:
+        x, xs = x32.to(torch.bfloat16), None
+    del x32
+    ids = torch.empty((T_max, k), dtype=torch.int32, device=device)
+    w = torch.empty((T_max, k), dtype=torch.float32, device=device)
+    out = torch.empty((T_max, H), dtype=torch.bfloat16, device=device)
+    points, result = cep.cep_calibrate(layer.plan, rho, list(rows), reps, x, xs, ids, w, out)
+    layer.close()
+    result.update({"config": cfg.name, "profile": points})
+    return result
+
+
 if __name__ == "__main__":
     name = sys.argv[1] if len(sys.argv) > 1 else "ep_shard"
-    print(json.dumps(calibrate(wl.CONFIGS[name])))
+    if len(sys.argv) > 2 and sys.argv[2] == "library":
+        print(json.dumps(calibrate_in_library(wl.CONFIGS[name])))
+    else:
+        print(json.dumps(calibrate(wl.CONFIGS[name])))

@@ -145,6 +145,7 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
 cudaError_t launch_combine(const BatchDesc& batch, const cep_config& cfg, const LayoutPtrs& lp,
                            const void* y, const void* addend, void* out, cudaStream_t s, int64_t* launches);
 cudaError_t launch_route(const float* logits, int T, int E_g, int k, int32_t* ids, float* weights, cudaStream_t s);
+cudaError_t launch_uniform_routing(int32_t* ids, float* weights, int T, int k, int k_loc, int E, cudaStream_t s);
 cudaError_t launch_gemm_simt(const GemmProblem& p, const void* a, const void* b, void* out,
                              const LayoutPtrs& lp, cudaStream_t s, int64_t* launches);
 cudaError_t launch_prepack(const cep_config& cfg, const void* w_gate, const void* w_up, const void* w_down,

@@ -57,6 +57,23 @@ route_kernel(const float* __restrict__ logits, int T, int E_g, int k, int32_t* _
 
 }  // namespace
 
+// Synthetic routing for the throughput profile: slot j < k_loc of token t goes to local expert (t*k_loc + j) mod E
+// (every expert gets the same number of rows), the remaining slots to experts of other ranks; weights 1/k_loc.
+__global__ void uniform_routing_kernel(int32_t* __restrict__ ids, float* __restrict__ w, int T, int k, int k_loc, int E) {
+  const long long n = (long long)T * k;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / k; const int j = (int)(i % k);
+    ids[i] = j < k_loc ? (int32_t)((t * k_loc + j) % E) : E + (j - k_loc);
+    w[i] = 1.f / (float)k_loc;
+  }
+}
+
+cudaError_t launch_uniform_routing(int32_t* ids, float* w, int T, int k, int k_loc, int E, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  uniform_routing_kernel<<<256, 256, 0, s>>>(ids, w, T, k, k_loc, E);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_route(const float* logits, int T, int E_g, int k, int32_t* ids, float* weights, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int warps_per_block = 8;

@@ -5,6 +5,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -144,6 +145,7 @@ struct cep_plan {
   Layout L;
   uint8_t* ws;
   int n_sms;
+  int active_streams;                           // round-robin over the first this-many streams / slots
   std::vector<cudaStream_t> streams;
   std::vector<Slot> slots;
   std::vector<cudaEvent_t> ready_evt;           // per chunk position
@@ -181,7 +183,7 @@ int launch_invocation(cep_plan* p) {
   const cep_config& c = p->cfg;
   const int idx = (int)p->inv.size();
   if (idx >= (int)p->inv_start.size()) return fail(p, CEP_ERR_CAPACITY, "more invocations than max_chunks");
-  const int slot_i = idx % c.n_streams;
+  const int slot_i = idx % p->active_streams;
   Slot& sl = p->slots[slot_i];
   cudaStream_t st = p->streams[slot_i];
   BatchDesc batch{};
@@ -312,7 +314,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   cep_plan* p = new (std::nothrow) cep_plan();
   if (!p) return fail(nullptr, CEP_ERR_ARG, "out of host memory");
   p->cfg = *cfg; p->L = L; p->ws = static_cast<uint8_t*>(workspace);
-  p->err[0] = 0; p->launches = 0;
+  p->err[0] = 0; p->launches = 0; p->active_streams = cfg->n_streams;
   p->have_weights = p->layer_open = p->flushed = p->readback_pending = p->ever_closed = false;
   p->host_status = nullptr; p->begin_evt = p->readback_evt = p->weights_evt = nullptr;
   p->out = nullptr; p->addend = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
@@ -575,7 +577,7 @@ int ffn_debug_export(cep_plan* p, int32_t inv, int32_t* counts, int32_t* offsets
   if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
   if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
   const Invocation& iv = p->inv[inv];
-  if ((int)p->inv.size() - inv > p->cfg.n_streams) return fail(p, CEP_ERR_STATE, "scratch slot of invocation %d was reused", inv);
+  if ((int)p->inv.size() - inv > p->active_streams) return fail(p, CEP_ERR_STATE, "scratch slot of invocation %d was reused", inv);
   CUDA_TRY(p, cudaEventSynchronize(iv.done));
   const Slot& sl = p->slots[iv.slot];
   const int E = p->cfg.n_experts_local;
@@ -592,6 +594,127 @@ int ffn_debug_export(cep_plan* p, int32_t inv, int32_t* counts, int32_t* offsets
   if (padded_offsets) memcpy(padded_offsets, po.data(), (E + 1) * 4);
   if (row_of_pair) CUDA_TRY(p, cudaMemcpy(row_of_pair, sl.lp.row_of_pair, (size_t)iv.n_tokens * p->cfg.top_k * 4, cudaMemcpyDeviceToHost));
   if (pair_of_row && po[E] > 0) CUDA_TRY(p, cudaMemcpy(pair_of_row, sl.lp.pair_of_row, (size_t)po[E] * 4, cudaMemcpyDeviceToHost));
+  return CEP_OK;
+}
+
+int ffn_set_active_streams(cep_plan* p, int32_t n) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (p->layer_open) return fail(p, CEP_ERR_STATE, "the number of active streams cannot change while a layer call is open");
+  if (n < 1 || n > p->cfg.n_streams) return fail(p, CEP_ERR_ARG, "active streams must be in 1..%d", p->cfg.n_streams);
+  p->active_streams = n;
+  return CEP_OK;
+}
+
+static float median_of(std::vector<float>& v) {
+  std::sort(v.begin(), v.end());
+  const size_t n = v.size();
+  return n == 0 ? -1.f : (n & 1) ? v[n / 2] : 0.5f * (v[n / 2 - 1] + v[n / 2]);
+}
+
+int cep_calibrate(cep_plan* p, float rho, const int32_t* rows_per_expert, int32_t n_points, int32_t reps,
+                  const void* tokens, const void* token_scales, int32_t* ids, float* weights, void* out,
+                  cep_profile_point* points, cep_calibration* res) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!rows_per_expert || !tokens || !ids || !weights || !out || !points || !res) return fail(p, CEP_ERR_ARG, "a calibration pointer is NULL");
+  if (!(rho > 0.f && rho <= 1.f) || n_points < 1 || reps < 1 || reps > 100) return fail(p, CEP_ERR_ARG, "need 0 < rho <= 1, n_points >= 1, 1 <= reps <= 100");
+  if (p->layer_open) return fail(p, CEP_ERR_STATE, "cep_calibrate while a layer call is open");
+  if (!p->have_weights) return fail(p, CEP_ERR_STATE, "cep_calibrate before moe_load_weights");
+  if (!p->cfg.profile_kernels) return fail(p, CEP_ERR_STATE, "cep_calibrate needs a plan made with profile_kernels != 0");
+  const cep_config saved = p->cfg;
+  const int saved_active = p->active_streams;
+  const int E = saved.n_experts_local, k = saved.top_k, k_loc = k < E ? k : E;
+  for (int i = 0; i < n_points; ++i) {
+    if (rows_per_expert[i] < 1 || (i > 0 && rows_per_expert[i] <= rows_per_expert[i - 1]))
+      return fail(p, CEP_ERR_ARG, "rows_per_expert must be positive and ascending");
+  }
+  auto tokens_for = [&](long long rows) { long long t = rows * E / k_loc; return t < 1 ? 1ll : t; };
+  const long long T_max = tokens_for(rows_per_expert[n_points - 1]);
+  if (T_max > saved.max_tokens) return fail(p, CEP_ERR_CAPACITY, "largest point needs %lld tokens, plan made for %d", T_max, saved.max_tokens);
+  cudaStream_t s0 = p->streams[0];
+  cudaEvent_t ea = nullptr, eb = nullptr;
+  int rc = CEP_OK;
+  const size_t act_row = (size_t)saved.hidden * (dtype_is_bytes(saved.dtype) ? 1 : 2);
+  const size_t scale_row = saved.dtype == CEP_BF16 ? 0 : (size_t)saved.hidden / kQuantBlock * 4;   // bytes of scales per token
+  auto restore = [&]() {
+    p->cfg.mode = saved.mode; p->cfg.threshold_pairs = saved.threshold_pairs; p->active_streams = saved_active;
+    if (ea) cudaEventDestroy(ea);
+    if (eb) cudaEventDestroy(eb);
+  };
+#define CAL_TRY(call) do { rc = (call); if (rc != CEP_OK) { restore(); return rc; } } while (0)
+#define CAL_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { restore(); \
+    return fail(p, CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); } } while (0)
+  CAL_CUDA(launch_uniform_routing(ids, weights, (int)T_max, k, k_loc, E, s0));
+  CAL_CUDA(cudaEventCreate(&ea));
+  CAL_CUDA(cudaEventCreate(&eb));
+  // ---- the profile: one synchronous invocation per point
+  p->cfg.mode = CEP_MODE_SYNC;
+  float peak = 0.f;
+  for (int i = 0; i < n_points; ++i) {
+    const int T = (int)tokens_for(rows_per_expert[i]);
+    std::vector<float> ffn, layer;
+    for (int r = 0; r < reps + 2; ++r) {
+      CAL_TRY(ffn_begin(p, out, T, 1));
+      CAL_TRY(ffn_submit_chunk(p, 0, 0, T, tokens, token_scales, ids, weights, (int64_t)T * k_loc, s0));
+      CAL_TRY(combine(p, s0));
+      CAL_CUDA(cudaStreamSynchronize(s0));
+      CAL_TRY(ffn_status(p));
+      cep_invocation_info info;
+      CAL_TRY(ffn_query(p, 0, &info));
+      if (r >= 2) { ffn.push_back(info.gemm1_ms + info.gemm2_ms); layer.push_back(info.elapsed_ms); }
+    }
+    cep_profile_point& pt = points[i];
+    pt.rows_per_expert = rows_per_expert[i]; pt.n_tokens = T; pt.expert_tokens = (int64_t)T * k_loc;
+    pt.ffn_ms = median_of(ffn); pt.layer_ms = median_of(layer);
+    pt.tflops = pt.ffn_ms > 0.f ? (float)(6.0 * saved.hidden * saved.inter * (double)pt.expert_tokens / (pt.ffn_ms * 1e-3) / 1e12) : 0.f;
+    pt.eta = 0.f;
+    if (pt.tflops > peak) peak = pt.tflops;
+  }
+  res->rho = rho; res->peak_tflops = peak; res->theta_pairs = points[n_points - 1].expert_tokens;
+  res->theta_rows_per_expert = points[n_points - 1].rows_per_expert;
+  for (int i = 0; i < n_points; ++i) points[i].eta = peak > 0.f ? points[i].tflops / peak : 0.f;
+  for (int i = 0; i < n_points; ++i)
+    if (points[i].eta >= rho) { res->theta_pairs = points[i].expert_tokens; res->theta_rows_per_expert = points[i].rows_per_expert; break; }
+  // ---- stream probe: a chain of theta-sized invocations, all chunks present, 1..S active streams
+  for (int s = 0; s < 16; ++s) res->stream_ms[s] = -1.f;
+  res->best_streams = 0; res->probe_invocations = 0;
+  const int T_theta = (int)tokens_for(res->theta_rows_per_expert);
+  int n_inv = (int)(T_max / T_theta);
+  if (n_inv > 8) n_inv = 8;
+  if (n_inv > saved.max_chunks) n_inv = saved.max_chunks;
+  if (n_inv >= 2 && saved.n_streams > 1) {
+    res->probe_invocations = n_inv;
+    p->cfg.mode = CEP_MODE_STREAMFFN;
+    p->cfg.threshold_pairs = (int64_t)T_theta * k_loc;
+    float best = -1.f;
+    for (int s = 1; s <= saved.n_streams; ++s) {
+      p->active_streams = s;
+      std::vector<float> ms;
+      for (int r = 0; r < reps + 2; ++r) {
+        CAL_CUDA(cudaEventRecord(ea, s0));
+        CAL_TRY(ffn_begin(p, out, n_inv * T_theta, n_inv));
+        for (int c = 0; c < n_inv; ++c) {
+          const uint8_t* tk = static_cast<const uint8_t*>(tokens) + (size_t)c * T_theta * act_row;
+          const uint8_t* sc = token_scales ? static_cast<const uint8_t*>(token_scales) + (size_t)c * T_theta * scale_row : nullptr;
+          CAL_TRY(ffn_submit_chunk(p, c, c * T_theta, T_theta, tk, sc, ids + (size_t)c * T_theta * k,
+                                   weights + (size_t)c * T_theta * k, (int64_t)T_theta * k_loc, s0));
+        }
+        CAL_TRY(combine(p, s0));
+        CAL_CUDA(cudaEventRecord(eb, s0));
+        CAL_CUDA(cudaStreamSynchronize(s0));
+        CAL_TRY(ffn_status(p));
+        float t = 0.f;
+        CAL_CUDA(cudaEventElapsedTime(&t, ea, eb));
+        if (r >= 2) ms.push_back(t);
+      }
+      res->stream_ms[s - 1] = median_of(ms);
+      if (best < 0.f || res->stream_ms[s - 1] < best) best = res->stream_ms[s - 1];
+    }
+    for (int s = 1; s <= saved.n_streams; ++s)
+      if (res->stream_ms[s - 1] <= 1.02f * best) { res->best_streams = s; break; }
+  }
+#undef CAL_TRY
+#undef CAL_CUDA
+  restore();
   return CEP_OK;
 }
 
