@@ -305,9 +305,16 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         tc_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN + col0), va);
         tc_wait_ld();
       }
+      // the scales of K block kb+1 are fetched while block kb is promoted: their L2 latency would otherwise sit
+      // in front of every block's first multiply-add
+      float sa_n = row_ok ? __ldg(sa_row) : 0.f, sw0_n = __ldg(sw0_p), sw1_n = __ldg(sw1_p);
       for (int kb = 0; kb < num_kb; ++kb) {
-        const float sa = row_ok ? __ldg(sa_row + kb) : 0.f;
-        const float s0 = sa * __ldg(sw0_p + kb), s1 = sa * __ldg(sw1_p + kb);
+        const float s0 = sa_n * sw0_n, s1 = sa_n * sw1_n;
+        if (kb + 1 < num_kb) {
+          sa_n = row_ok ? __ldg(sa_row + kb + 1) : 0.f;
+          sw0_n = __ldg(sw0_p + kb + 1);
+          sw1_n = __ldg(sw1_p + kb + 1);
+        }
         const uint32_t t_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN);
         tc_ld32(t_addr + (uint32_t)(col0 + 32), vb);
         CEP_FMA_CHUNK(va, 0, s0);
