@@ -199,7 +199,7 @@ CEP_API int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts_g
  *   chunk_id       0..n_chunks_expected-1, each exactly once, any order
  *   token_offset   first token (row of `out`) this chunk covers
  *   tokens         [device] bf16 [n,H]  |  e4m3 [n,H]
- *   token_scales   [device] fp32 [n,H/128] for fp8; uint8 ue8m0 [n,H/32] for mxfp4; else NULL
+ *   token_scales   [device] fp32 [n,H/128] for fp8; uint8 ue8m0 [n,H/32] for mxfp4 (4-byte aligned); else NULL
  *   topk_ids       [device] int32 [n,k] global expert ids, distinct per token
  *   topk_weights   [device] fp32 [n,k]
  *   n_local_pairs  number of (token,slot) pairs with id < n_experts_local, as known from

@@ -105,3 +105,15 @@ def test_null_plan_is_rejected_without_touching_a_device():
     assert L.ffn_status(None) == -1
     assert L.moe_plan_destroy(None) == 0
     assert b"NULL" in L.cep_last_error(None)
+    assert L.ffn_set_active_streams(None, 1) == -1
+    assert L.cep_calibrate(None, 0.9, None, 0, 0, None, None, None, None, None, None, None) == -1
+
+
+def test_microscaling_config_is_validated_on_the_host():
+    ok = cep.CepConfig(512, 256, 8, 8, 2, 256, 2, cep.CEP_MXFP4_E4M3, 0, 2, 0, 0, 0)
+    assert cep.moe_plan_workspace_bytes(ok) > 0
+    bf16 = cep.CepConfig(512, 256, 8, 8, 2, 256, 2, cep.CEP_BF16, 0, 2, 0, 0, 0)
+    # packed weights: a nibble + 1/32 scale byte per element against two bytes
+    assert cep.moe_packed_weight_bytes(ok) < cep.moe_packed_weight_bytes(bf16) // 3
+    with pytest.raises(cep.CepError):
+        cep.moe_plan_workspace_bytes(cep.CepConfig(512, 256, 8, 8, 2, 256, 2, 3, 0, 2, 0, 0, 0))     # unknown dtype
