@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 CFG = wl.MoEConfig("cal", 1, T=2048, H=1024, I=512, E_global=16, E_local=8, k=4, chunks=(2048,))
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "mxfp4"])
+@pytest.mark.parametrize("dtype", ["bf16", "fp8", "mxfp4"])
 def test_library_calibration_profile_and_threshold(dtype):
     cfg = wl.scaled(CFG, dtype=dtype)
     rows = (16, 64, 256, 1024)
