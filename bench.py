@@ -335,11 +335,12 @@ def main():
             sets.append({"dx": torch.empty_like(inp.x), "did": torch.empty_like(inp.topk_ids), "dw": torch.empty_like(inp.topk_w),
                          "dxs": None if inp.x_scale is None else torch.empty_like(inp.x_scale),
                          "out": torch.empty_like(out), "hout": torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory(),
-                         "free": torch.cuda.Event()})
+                         "in_free": torch.cuda.Event(), "out_free": torch.cuda.Event()})
         rstreams = [torch.cuda.Stream() for _ in chunks]
         main = torch.cuda.current_stream()
         for b_ in sets:
-            b_["free"].record(main)
+            b_["in_free"].record(main)
+            b_["out_free"].record(main)
 
         # chunks are consumed as they land (Async+streamFFN, theta = two chunks' worth of pairs) and every
         # invocation's output rows are copied back as soon as that invocation has written them
@@ -354,6 +355,7 @@ def main():
                                   mode=cep.CEP_MODE_SYNC, n_streams=2, gemm_impl=args.gemm_impl)
         sync_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
         d2h = torch.cuda.Stream()
+        free_s = torch.cuda.Stream()
 
         def e2e_step(i, overlap, e2e_layer=e2e_layer):
             b_ = sets[i % 2 if overlap else 0]
@@ -363,7 +365,7 @@ def main():
             for c, (o, n) in enumerate(zip(inp.chunk_offsets, cfg.chunks)):
                 st = rstreams[c]
                 if overlap:
-                    st.wait_event(b_["free"])           # the layer call that last used this buffer set is complete
+                    st.wait_event(b_["in_free"])        # the call that last used these input buffers has consumed them
                 else:
                     st.wait_stream(main)                # one layer call at a time
                 with torch.cuda.stream(st):
@@ -372,6 +374,8 @@ def main():
                     dw[o:o + n].copy_(hw[o:o + n], non_blocking=True)
                     if dxs is not None:
                         dxs[o:o + n].copy_(hxs[o:o + n], non_blocking=True)
+                if overlap:
+                    st.wait_event(b_["out_free"])       # ... and its output rows have left the output buffer
                 cep.ffn_submit_chunk(e2e_layer.plan, c, o, n, dx[o:o + n], None if dxs is None else dxs[o:o + n],
                                      did[o:o + n], dw[o:o + n], ch_pairs[c], st)
                 if c == len(chunks) - 1:
@@ -386,9 +390,12 @@ def main():
                     with torch.cuda.stream(d2h):
                         hout[lo:hi].copy_(dout[lo:hi], non_blocking=True)
                     seen += 1
+            for j in range(cep.ffn_num_invocations(e2e_layer.plan)):
+                cep.ffn_wait_invocation(e2e_layer.plan, j, free_s)
+            b_["in_free"].record(free_s)                # every invocation of this call has finished reading its inputs
             cep.combine(e2e_layer.plan, main)
             main.wait_stream(d2h)
-            b_["free"].record(main)
+            b_["out_free"].record(main)
 
         def e2e_run(overlap, layer_):
             for i in range(4):

@@ -18,6 +18,7 @@ namespace {
 
 char g_error[256] = "";
 constexpr int kGuardByte = 0xA5;
+constexpr size_t kStatusBlockBytes = 256;        // one status block (kStWords int32) per layer-call parity
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -152,8 +153,13 @@ struct cep_plan {
   std::vector<Invocation> inv;
   std::vector<cudaEvent_t> inv_start, inv_done; // pools, one per possible invocation
   std::vector<cudaEvent_t> inv_mark;            // 4 per possible invocation (profile_kernels)
-  cudaEvent_t begin_evt, readback_evt, weights_evt;
-  bool have_weights, layer_open, flushed, readback_pending, ever_closed;
+  // Two status blocks, used by alternate layer calls: a call clears its block without waiting for the previous
+  // call's read-back (a small device-to-host copy that can sit behind the caller's own output copies in the copy
+  // engine's queue), only for the read-back of the call before that.
+  cudaEvent_t begin_evt, readback_evt[2], weights_evt;
+  int status_idx;                               // block of the current / last layer call
+  bool readback_pending[2];
+  bool have_weights, layer_open, flushed, ever_closed;
   uint8_t* w13p; uint8_t* w2p;
   void* s13p; void* s2p;                        // fp8, mxfp4: packed weight scales
   GemmTensorMap tm_b1, tm_b2;
@@ -163,7 +169,7 @@ struct cep_plan {
   std::vector<char> chunk_seen;
   std::vector<PendingChunk> pending;
   int64_t pending_pairs;
-  int32_t* host_status;                         // pinned
+  int32_t* host_status;                         // pinned, two blocks of kStWords
   int64_t launches;
   char err[256];
 };
@@ -315,18 +321,20 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   if (!p) return fail(nullptr, CEP_ERR_ARG, "out of host memory");
   p->cfg = *cfg; p->L = L; p->ws = static_cast<uint8_t*>(workspace);
   p->err[0] = 0; p->launches = 0; p->active_streams = cfg->n_streams;
-  p->have_weights = p->layer_open = p->flushed = p->readback_pending = p->ever_closed = false;
-  p->host_status = nullptr; p->begin_evt = p->readback_evt = p->weights_evt = nullptr;
+  p->have_weights = p->layer_open = p->flushed = p->ever_closed = false;
+  p->readback_pending[0] = p->readback_pending[1] = false; p->status_idx = 0;
+  p->host_status = nullptr; p->begin_evt = p->readback_evt[0] = p->readback_evt[1] = p->weights_evt = nullptr;
   p->out = nullptr; p->addend = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
   int dev = 0;
 #define PLAN_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
     fail(nullptr, CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); moe_plan_destroy(p); return CEP_ERR_CUDA; } } while (0)
   PLAN_TRY(cudaGetDevice(&dev));
   PLAN_TRY(cudaDeviceGetAttribute(&p->n_sms, cudaDevAttrMultiProcessorCount, dev));
-  PLAN_TRY(cudaHostAlloc(reinterpret_cast<void**>(&p->host_status), kStWords * sizeof(int32_t), cudaHostAllocDefault));
-  memset(p->host_status, 0, kStWords * sizeof(int32_t));
+  PLAN_TRY(cudaHostAlloc(reinterpret_cast<void**>(&p->host_status), 2 * kStWords * sizeof(int32_t), cudaHostAllocDefault));
+  memset(p->host_status, 0, 2 * kStWords * sizeof(int32_t));
   PLAN_TRY(cudaEventCreateWithFlags(&p->begin_evt, cudaEventDisableTiming));
-  PLAN_TRY(cudaEventCreateWithFlags(&p->readback_evt, cudaEventDisableTiming));
+  PLAN_TRY(cudaEventCreateWithFlags(&p->readback_evt[0], cudaEventDisableTiming));
+  PLAN_TRY(cudaEventCreateWithFlags(&p->readback_evt[1], cudaEventDisableTiming));
   PLAN_TRY(cudaEventCreateWithFlags(&p->weights_evt, cudaEventDisableTiming));
   for (int s = 0; s < cfg->n_streams; ++s) {
     cudaStream_t st;
@@ -375,7 +383,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   }
   if (L.guard) PLAN_TRY(cudaMemsetAsync(p->ws, kGuardByte, L.total, p->streams[0]));   // gaps keep this pattern
   // status word starts clean
-  PLAN_TRY(cudaMemsetAsync(p->ws + L.status, 0, kStWords * sizeof(int32_t), p->streams[0]));
+  PLAN_TRY(cudaMemsetAsync(p->ws + L.status, 0, 2 * kStatusBlockBytes, p->streams[0]));
   PLAN_TRY(cudaEventRecord(p->begin_evt, p->streams[0]));
   PLAN_TRY(cudaEventRecord(p->weights_evt, p->streams[0]));
 #undef PLAN_TRY
@@ -438,8 +446,13 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   if (n_chunks_expected > p->cfg.max_chunks) return fail(p, CEP_ERR_CAPACITY, "%d chunks, plan made for %d", n_chunks_expected, p->cfg.max_chunks);
   cudaStream_t s0 = p->streams[0];
   // the previous layer's status read-back must finish before the status word is cleared
-  if (p->readback_pending) CUDA_TRY(p, cudaStreamWaitEvent(s0, p->readback_evt, 0));
-  CUDA_TRY(p, cudaMemsetAsync(p->ws + p->L.status, 0, kStWords * sizeof(int32_t), s0));
+  p->status_idx ^= 1;
+  const int sb = p->status_idx;
+  // the read-back of the call that last used this status block must finish before the block is cleared
+  if (p->readback_pending[sb]) CUDA_TRY(p, cudaStreamWaitEvent(s0, p->readback_evt[sb], 0));
+  int32_t* status_dev = reinterpret_cast<int32_t*>(p->ws + p->L.status + (size_t)sb * kStatusBlockBytes);
+  for (Slot& sl : p->slots) sl.lp.status = status_dev;
+  CUDA_TRY(p, cudaMemsetAsync(status_dev, 0, kStWords * sizeof(int32_t), s0));
   CUDA_TRY(p, cudaEventRecord(p->begin_evt, s0));
   p->out = out; p->addend = nullptr; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
   p->n_submitted = 0; p->tokens_submitted = 0;
@@ -522,9 +535,11 @@ int combine(cep_plan* p, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
   for (const Invocation& iv : p->inv) CUDA_TRY(p, cudaStreamWaitEvent(st, iv.done, 0));
-  CUDA_TRY(p, cudaMemcpyAsync(p->host_status, p->ws + p->L.status, kStWords * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(p, cudaEventRecord(p->readback_evt, st));
-  p->readback_pending = true; p->ever_closed = true;
+  const int sb = p->status_idx;
+  CUDA_TRY(p, cudaMemcpyAsync(p->host_status + sb * kStWords, p->ws + p->L.status + (size_t)sb * kStatusBlockBytes,
+                              kStWords * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(p, cudaEventRecord(p->readback_evt[sb], st));
+  p->readback_pending[sb] = true; p->ever_closed = true;
   p->layer_open = false;
   return rc;
 }
@@ -532,12 +547,13 @@ int combine(cep_plan* p, void* stream) {
 int ffn_status(cep_plan* p) {
   if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
   if (!p->ever_closed || p->layer_open) return fail(p, CEP_ERR_STATE, "no closed layer call to report on");
-  cudaError_t q = cudaEventQuery(p->readback_evt);
+  const int32_t* hs = p->host_status + p->status_idx * kStWords;
+  cudaError_t q = cudaEventQuery(p->readback_evt[p->status_idx]);
   if (q == cudaErrorNotReady) return fail(p, CEP_ERR_STATE, "the stream given to combine has not completed yet");
   if (q != cudaSuccess) return fail(p, CEP_ERR_CUDA, "cudaEventQuery failed: %s", cudaGetErrorString(q));
-  if (p->host_status[kStTimeout]) return fail(p, CEP_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired");
-  if (p->host_status[kStBoundsViolation]) return fail(p, CEP_ERR_CAPACITY, "a row index left the scratch slot (more local pairs than planned)");
-  if (p->host_status[kStBadRouting]) return fail(p, CEP_ERR_BAD_ROUTING, "an expert id was outside [0, n_experts_global)");
+  if (hs[kStTimeout]) return fail(p, CEP_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired");
+  if (hs[kStBoundsViolation]) return fail(p, CEP_ERR_CAPACITY, "a row index left the scratch slot (more local pairs than planned)");
+  if (hs[kStBadRouting]) return fail(p, CEP_ERR_BAD_ROUTING, "an expert id was outside [0, n_experts_global)");
   return CEP_OK;
 }
 
@@ -728,7 +744,8 @@ int moe_plan_destroy(cep_plan* p) {
   for (cudaEvent_t e : p->inv_done) cudaEventDestroy(e);
   for (cudaEvent_t e : p->inv_mark) cudaEventDestroy(e);
   if (p->begin_evt) cudaEventDestroy(p->begin_evt);
-  if (p->readback_evt) { cudaEventSynchronize(p->readback_evt); cudaEventDestroy(p->readback_evt); }
+  for (int i = 0; i < 2; ++i)
+    if (p->readback_evt[i]) { cudaEventSynchronize(p->readback_evt[i]); cudaEventDestroy(p->readback_evt[i]); }
   if (p->weights_evt) cudaEventDestroy(p->weights_evt);
   for (cudaStream_t s : p->streams) cudaStreamDestroy(s);
   if (p->host_status) cudaFreeHost(p->host_status);
@@ -743,7 +760,8 @@ int cep_debug_wait_timeout(cep_plan* p, int32_t limit_ms, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));          // after this call's status reset
   CUDA_TRY(p, launch_wait_probe((unsigned long long)limit_ms * 1000000ull,
-                                reinterpret_cast<int32_t*>(p->ws + p->L.status), st, &p->launches));
+                                reinterpret_cast<int32_t*>(p->ws + p->L.status + (size_t)p->status_idx * kStatusBlockBytes), st,
+                                &p->launches));
   return CEP_OK;
 }
 
