@@ -653,6 +653,7 @@ int cep_calibrate(cep_plan* p, float rho, const int32_t* rows_per_expert, int32_
   const size_t scale_row = saved.dtype == CEP_BF16 ? 0 : (size_t)saved.hidden / kQuantBlock * 4;   // bytes of scales per token
   auto restore = [&]() {
     p->cfg.mode = saved.mode; p->cfg.threshold_pairs = saved.threshold_pairs; p->active_streams = saved_active;
+    if (p->layer_open) { p->pending.clear(); p->pending_pairs = 0; p->layer_open = false; }   // a probe call that failed half-way
     if (ea) cudaEventDestroy(ea);
     if (eb) cudaEventDestroy(eb);
   };
