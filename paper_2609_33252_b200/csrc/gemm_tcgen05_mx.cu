@@ -45,12 +45,13 @@ constexpr int B_TX = (BN / 2) * BKE / 2;               // bytes the TMA engine c
 constexpr int SFA_STAGE = kSfAtomBytes;                // 128 rows x 4 scale blocks
 constexpr int SFB_STAGE = 2 * kSfAtomBytes;            // 256 weight rows x 4 scale blocks
 constexpr int kStages = 6;                             // K=128 slabs of operands in shared memory
-// Slabs are handed between producer and MMA warp two at a time: one barrier round trip (wait, fence, commit) per
-// eight MMAs instead of four.  Measured on the 7168x2048 expert shapes: GEMM1 2260 -> 2390 TFLOP/s, GEMM2 2206 ->
-// 2280; three at a time helps the long-K GEMM1 a little more but leaves the K=2048 GEMM2 only two rounds deep.
-constexpr int kGroup = 2;
-constexpr int kRounds = kStages / kGroup;
-static_assert(kStages % kGroup == 0, "slabs per round");
+// Slabs are handed between producer and MMA warp several at a time: one barrier round trip (wait, fence, commit) per
+// eight or twelve MMAs instead of four.  Measured on the 7168x2048 expert shapes: two at a time GEMM1 2260 -> 2390
+// TFLOP/s, GEMM2 2206 -> 2280; three at a time helps the K=7168 GEMM1 a little more (2420-2490) but leaves the
+// K=2048 GEMM2 only two rounds deep (2100-2150).
+// The group size is a template parameter: 3 for long K loops (at least kLongK slabs), 2 otherwise.
+constexpr int kMaxRounds = 3;
+constexpr int kLongK = 24;
 constexpr int kThreads = 384;
 constexpr int kEpiWarp0 = 4, kEpiWarps = 8;
 constexpr int kTmemCols = 512;
@@ -63,7 +64,7 @@ constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE + SFA_STAGE + SFB_STAGE)
 constexpr uint32_t kStageTx = 2u * (A_STAGE + B_TX + SFA_STAGE + SFB_STAGE);   // both CTAs' bytes, counted at the leader
 
 struct __align__(8) Bars {
-  uint64_t full[kRounds], empty[kRounds];
+  uint64_t full[kMaxRounds], empty[kMaxRounds];
   uint64_t acc_full, acc_empty;
   uint64_t sched_full[kRing], sched_empty[kRing];
   int32_t sched_tile[kRing];
@@ -135,7 +136,7 @@ __device__ __forceinline__ float mx_inv_scale(uint32_t code) {
   return code <= 253u ? __uint_as_float((254u - code) << 23) : __uint_as_float(0x00400000u);
 }
 
-template <bool kSwiglu>
+template <bool kSwiglu, int kGroup>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                        const __grid_constant__ CUtensorMap tm_sfa, const __grid_constant__ CUtensorMap tm_sfb,
@@ -147,6 +148,8 @@ grouped_gemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                        int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   pdl_enter();
+  constexpr int kRounds = kStages / kGroup;
+  static_assert(kStages % kGroup == 0 && kRounds <= kMaxRounds, "slabs per round");
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem_a + kStages * A_STAGE;
@@ -429,9 +432,10 @@ int g_clusters = -1;
 
 cudaError_t setup(int n_sms) {
   if (g_clusters >= 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_mx_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(grouped_gemm_mx_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaSuccess;
+#define CEP_MX_ATTR(SW, G) if (e == cudaSuccess) e = cudaFuncSetAttribute(grouped_gemm_mx_kernel<SW, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  CEP_MX_ATTR(true, 2) CEP_MX_ATTR(true, 3) CEP_MX_ATTR(false, 2) CEP_MX_ATTR(false, 3)
+#undef CEP_MX_ATTR
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
@@ -440,7 +444,7 @@ cudaError_t setup(int n_sms) {
   cfg.gridDim = dim3(n_sms & ~1, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes; cfg.attrs = attr; cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_mx_kernel<true>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_mx_kernel<true, 2>, &cfg);
   if (e != cudaSuccess) return e;
   g_clusters = n;
   return cudaSuccess;
@@ -535,16 +539,15 @@ cudaError_t launch_gemm_mx(const GemmProblem& p, const GemmTensorMap& tm_a, cons
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
   const CUtensorMap& sa = reinterpret_cast<const CUtensorMap&>(tm_sfa);
   const CUtensorMap& sb = reinterpret_cast<const CUtensorMap&>(tm_sfb);
-  if (p.swiglu)
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_mx_kernel<true>, a, b, sa, sb, num_kb, n_blocks_n, n_group, p.n_experts,
-                           n_out_cols, p.out_ld, (uint8_t*)out, (uint8_t*)out_sf, (__nv_bfloat16*)nullptr,
-                           (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
-                           counter, lp.status);
-  else
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_mx_kernel<false>, a, b, sa, sb, num_kb, n_blocks_n, n_group, p.n_experts,
-                           n_out_cols, p.out_ld, (uint8_t*)nullptr, (uint8_t*)nullptr, (__nv_bfloat16*)out,
-                           (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
-                           counter, lp.status);
+#define CEP_MX_LAUNCH(SW, G)                                                                                           \
+  cudaLaunchKernelEx(&cfg, grouped_gemm_mx_kernel<SW, G>, a, b, sa, sb, num_kb, n_blocks_n, n_group, p.n_experts,          \
+                     n_out_cols, p.out_ld, SW ? (uint8_t*)out : (uint8_t*)nullptr, SW ? (uint8_t*)out_sf : (uint8_t*)nullptr, \
+                     SW ? (__nv_bfloat16*)nullptr : (__nv_bfloat16*)out, (const int32_t*)lp.tile_prefix,                   \
+                     (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, counter, lp.status)
+  const bool long_k = num_kb >= kLongK;
+  if (p.swiglu) e = long_k ? CEP_MX_LAUNCH(true, 3) : CEP_MX_LAUNCH(true, 2);
+  else e = long_k ? CEP_MX_LAUNCH(false, 3) : CEP_MX_LAUNCH(false, 2);
+#undef CEP_MX_LAUNCH
   *launches += 1;
   return e;
 }
