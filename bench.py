@@ -447,7 +447,9 @@ def main():
     # (cap reported active, clock well below maximum, or more than a second of back-to-back steps)
     sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
     capped = "sw_power_cap" in ((clocks or {}).get("reasons") or [])
-    sustained = capped or (total_ms > 1000.0) or bool(sm and smx and sm < 0.9 * smx)
+    # (the power controller needs on the order of 100 ms of load before it pulls the clocks down: a timed region
+    # shorter than that ran at burst clocks whatever the sampled flags say)
+    sustained = total_ms > 100.0 and (capped or total_ms > 1000.0 or bool(sm and smx and sm < 0.9 * smx))
     peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     nominal_tf = NOMINAL_BF16_TFLOPS
     if cfg.dtype in ("fp8", "mxfp4"):   # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2);
