@@ -87,6 +87,8 @@ CONFIGS = {
                             chunks=(160, 96), dtype="mxfp4"),
     "mxfp4_shard_small": MoEConfig("mxfp4_shard_small", 5, T=2048, H=7168, I=2048, E_global=64, E_local=8, k=8,
                                    chunks=tuple(_equal_chunks(2048, 8)), dtype="mxfp4", zipf_s=1.1),
+    "mxfp4_straggler": MoEConfig("mxfp4_straggler", 5, T=16384, H=7168, I=2048, E_global=256, E_local=32, k=8,
+                                 chunks=(1404,) * 7 + (16384 - 7 * 1404,), dtype="mxfp4", zipf_s=1.1, straggler_last=True),
     "mxfp4_shard": MoEConfig("mxfp4_shard", 5, T=16384, H=7168, I=2048, E_global=256, E_local=32, k=8,
                              chunks=tuple(_equal_chunks(16384, 8)), dtype="mxfp4", zipf_s=1.1),
 }
