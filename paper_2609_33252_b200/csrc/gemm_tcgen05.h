@@ -30,7 +30,9 @@ int gemm_pair_clusters();
 
 // Block-scaled e4m3 variant.  a_scales [rows, K/128], b_scales [E, N/128, K/128] fp32.  With p.swiglu the output is
 // e4m3 codes [rows, N/2] plus out_scales [rows, N/256]; otherwise bf16 [rows, N].  pair != 0: CTA pairs on 256x256
-// tiles (weight map with a 128-row box); pair == 0: one CTA per 128x256 tile (256-row box).
+// tiles; pair == 0: one CTA per 128x256 tile.  The weight map's box has gemm_fp8_box_rows(pair) rows (the weight
+// rows one CTA loads per stage).
+int gemm_fp8_box_rows(int pair);
 cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                             const float* a_scales, const float* b_scales, void* out, float* out_scales,
                             const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches);

@@ -7,14 +7,24 @@
 // scaling.  Each K block is therefore multiplied on its own into a scratch accumulator in tensor memory
 // (tcgen05.mma kind::f8f6f4, fp32 accumulate, two scratch buffers in flight), and eight "promotion"
 // warps pull every partial product out of tensor memory and add it, scaled, into fp32 accumulators
-// they hold in registers (128 per thread).  The same warps then run the epilogue:
+// they hold in registers (128 per thread).
+//
+// What paces such a loop is the thread that issues the MMAs: every tcgen05 instruction (mma, commit) and
+// every barrier wait costs that one thread 60-100 cycles, and a K block here needs two waits (operands
+// landed, scratch buffer free) on top of its four MMAs, against 512 cycles of tensor work.  So the issue
+// is split over TWO threads, one per scratch buffer: K blocks alternate between them, each thread waits,
+// issues and commits for its own buffer only, and since every K block goes to its own buffer and the
+// promotion warps consume the buffers in K order, the result does not depend on how the two threads'
+// MMAs interleave in the tensor pipe.  One commit per K block serves both as "operands consumed" for the
+// TMA producer and as "partial product ready" for the promotion warps (barrier done[stage]).
+// The promotion warps also run the epilogue:
 //   GEMM1: SiLU(gate)*up, per-row amax over the tile's 128 columns, scale = amax/448, e4m3 codes
 //          (round-to-nearest-even, saturating) + the scale: the "activation and quantization" step
 //          between the two expert GEMMs (Appendix "Grouped FFN invocations")
 //   GEMM2: bf16
-// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer (leader CTA), warp 2 tile scheduler
-// (leader CTA), warps 4-11 promotion + epilogue.  Tiles come from a global counter, as in the bf16
-// kernel.  All waits are bounded.
+// Roles (384 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of even / odd K blocks (leader CTA),
+// warp 2 tile scheduler (leader CTA), warps 4-11 promotion + epilogue.  Tiles come from a global
+// counter, as in the bf16 kernel.  All waits are bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -33,41 +43,59 @@ constexpr int A_STAGE = BM * BKB;                      // 16 KiB
 // kPair: CTA pairs (256x256 tiles, each CTA loads half of the weight tile, 6 stages of 32 KiB);
 // !kPair: one CTA per 128x256 tile (whole weight tile per CTA, 4 stages of 48 KiB): every hand-off
 // between the MMA warp and the promotion warps stays inside the SM
+constexpr int kBarBytes = 512;
+constexpr int kPromoWarp0 = 4, kPromoWarps = 8;
+constexpr int kStoreStage = 2048;                      // per promotion warp: 32 rows x 64 bytes of output on their way to global memory
 template <bool kPair> struct Geo {
   static constexpr int kStages = kPair ? 6 : 4;
   static constexpr int B_STAGE = (kPair ? BN / 2 : BN) * BKB;
-  static constexpr int kRingReaders = kPair ? 19 : 10;    // producer, MMA, 8 promotion warps (+ peer: producer, 8)
+  static constexpr int kRingReaders = kPair ? 20 : 11;    // producer, 2 MMA issuers, 8 promotion warps (+ peer: producer, 8)
   static constexpr int kPartArrivals = kPair ? 16 : 8;
-  static constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE) + 256 + (1024 + 1) * 4 + 2 * 2 * BM * 4 + 1024;
+  static constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE) + kBarBytes + (1024 + 1) * 4 + 12 + 2 * 2 * BM * 4 +
+                                    kPromoWarps * kStoreStage + 1024;
 };
 constexpr int kMaxStages = 6;
 constexpr int kThreads = 384;
-constexpr int kPromoWarp0 = 4, kPromoWarps = 8;
 constexpr int kTmemCols = 512;
 constexpr int kMaxExperts = 1024;
 constexpr int kRing = 4;
 constexpr int kTilePoison = -2;
 
 struct __align__(8) Bars {
-  uint64_t full[kMaxStages], empty[kMaxStages];
-  uint64_t part_full[2], part_empty[2];               // scratch accumulators in tensor memory
+  uint64_t full[kMaxStages];                          // operands of the stage have landed
+  uint64_t done[kMaxStages];                          // the stage's MMAs have completed: operands consumed, partial ready
+  uint64_t part_empty[2];                             // scratch accumulators in tensor memory read out
   uint64_t sched_full[kRing], sched_empty[kRing];
   uint64_t amax_bar[4];                               // per lane group: the two warps sharing its rows
-  int32_t sched_tile[kRing];
+  int32_t sched_tile[kRing][8];                       // a handed-out tile, decoded: see TileInfo
   uint32_t tmem_base;
   int abort_flag;
 };
-static_assert(sizeof(Bars) <= 256, "barrier block");
+static_assert(sizeof(Bars) <= kBarBytes, "barrier block");
+static_assert(BKB == 128 && Geo<true>::kStages % 2 == 0 && Geo<false>::kStages % 2 == 0, "a stage always pairs with the same scratch buffer");
+
+// What the scheduler thread publishes per tile, so that no other role has to search the tile table or
+// touch global memory at a tile boundary.
+struct TileInfo {
+  int tile;                    // linear index, -1: no more tiles
+  int expert, m_block, n_block;
+  int count;                   // rows of the expert
+  int poff;                    // first (tile-aligned) row of the expert's group
+};
 
 struct Ring {
   int slot = 0; uint32_t phase = 0;
-  __device__ __forceinline__ int next(Bars* b, bool is_peer, volatile int* abort_flag, int32_t* status) {
+  __device__ __forceinline__ TileInfo next(Bars* b, bool is_peer, volatile int* abort_flag, int32_t* status) {
+    TileInfo ti;
+    ti.tile = -1; ti.expert = ti.m_block = ti.n_block = ti.count = ti.poff = 0;
     const uint32_t bar = smem_u32(&b->sched_full[slot]);
     const bool ok = is_peer ? mbar_wait_acq_cluster(bar, phase, abort_flag, status) : mbar_wait(bar, phase, abort_flag, status);
-    if (!ok) return -1;
-    const int t = b->sched_tile[slot];
-    if (t < -1) { atomicExch(&status[kStDetail], 0x5C4ED); atomicExch(&status[kStTimeout], 1); *abort_flag = 1; return -1; }
-    return t;
+    if (!ok) return ti;
+    const int4 v = *reinterpret_cast<const int4*>(&b->sched_tile[slot][0]);
+    const int2 w = *reinterpret_cast<const int2*>(&b->sched_tile[slot][4]);
+    if (v.x < -1) { atomicExch(&status[kStDetail], 0x5C4ED); atomicExch(&status[kStTimeout], 1); *abort_flag = 1; return ti; }
+    ti.tile = v.x; ti.expert = v.y; ti.m_block = v.z; ti.n_block = v.w; ti.count = w.x; ti.poff = w.y;
+    return ti;
   }
   template <bool kPair>
   __device__ __forceinline__ void done(Bars* b, bool signal) {
@@ -79,13 +107,31 @@ struct Ring {
   }
 };
 
-__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// kAcc (0: overwrite the accumulator, 1: add to it) is an immediate, so the issuing thread spends no instruction on it
+template <int kAcc>
+__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "n"(kAcc) : "memory");
 }
-__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+template <int kAcc>
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "n"(kAcc) : "memory");
+}
+// the four K=32 MMAs of one 128-deep K block (a descriptor advances by 32 bytes = 2 units per MMA)
+template <bool kPair>
+__device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  if (kPair) {
+    tc_mma_f8_pair<0>(d_tmem, adesc, bdesc, idesc);
+    tc_mma_f8_pair<1>(d_tmem, adesc + 2, bdesc + 2, idesc);
+    tc_mma_f8_pair<1>(d_tmem, adesc + 4, bdesc + 4, idesc);
+    tc_mma_f8_pair<1>(d_tmem, adesc + 6, bdesc + 6, idesc);
+  } else {
+    tc_mma_f8<0>(d_tmem, adesc, bdesc, idesc);
+    tc_mma_f8<1>(d_tmem, adesc + 2, bdesc + 2, idesc);
+    tc_mma_f8<1>(d_tmem, adesc + 4, bdesc + 4, idesc);
+    tc_mma_f8<1>(d_tmem, adesc + 6, bdesc + 6, idesc);
+  }
 }
 // kind::f8f6f4: fp32 accumulate, e4m3 x e4m3 (format code 0), both operands K-major
 __host__ __device__ constexpr uint32_t make_idesc_e4m3(int m, int n) {
@@ -112,6 +158,25 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
   return r;
 }
 
+// A warp holds 64 bytes of output per lane (lane = row).  Written to global memory directly, every store
+// instruction would touch 32 rows with 16 bytes each; staged through 2 KiB of shared memory (16-byte chunks
+// swizzled by row so that neither side has bank conflicts) each instruction covers 64 contiguous bytes of 8 rows.
+// Rows at or beyond n_rows are not stored.  dst = address of row 0, row_stride in bytes.
+__device__ __forceinline__ void store_rows_64B(uint8_t* stage, int lane, const uint4 (&ch)[4], uint8_t* dst,
+                                               size_t row_stride, int n_rows) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) = ch[q];
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + (lane >> 2), c = lane & 3;
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 64 + ((c ^ ((r >> 1) & 3)) << 4));
+    if (r < n_rows) *reinterpret_cast<uint4*>(dst + (size_t)r * row_stride + c * 16) = v;
+  }
+  __syncwarp();
+}
+
 template <bool kSwiglu, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -131,19 +196,20 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + kStages * A_STAGE;
   Bars* bars = reinterpret_cast<Bars*>(smem + kStages * (A_STAGE + B_STAGE));
-  int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kStages * (A_STAGE + B_STAGE) + 256);
-  float* s_amax = reinterpret_cast<float*>(pair_prefix + kMaxExperts + 1);           // [tile parity][half][128]
+  int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kStages * (A_STAGE + B_STAGE) + kBarBytes);
+  float* s_amax = reinterpret_cast<float*>(pair_prefix + kMaxExperts + 4);           // [tile parity][half][128]
+  uint8_t* s_store = reinterpret_cast<uint8_t*>(s_amax + 2 * 2 * BM);                // [promotion warp][kStoreStage]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = kPair ? cluster_ctarank() : 0u;
   const bool is_peer = rank != 0;
   volatile int* abort_flag = &bars->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->part_full[s]), 1); mbar_init(smem_u32(&bars->part_empty[s]), Geo<kPair>::kPartArrivals); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->done[s]), 1); }
+    for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&bars->part_empty[s]), Geo<kPair>::kPartArrivals);
     for (int s = 0; s < kRing; ++s) {
       mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), Geo<kPair>::kRingReaders);
-      bars->sched_tile[s] = kTilePoison;
+      bars->sched_tile[s][0] = kTilePoison;
     }
     for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars->amax_bar[s]), 2);
     bars->abort_flag = 0;
@@ -185,15 +251,13 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       bool ok = true;
       Ring rd;
       for (; ok;) {
-        const int tile = rd.next(bars, is_peer, abort_flag, status);
+        const TileInfo tc = rd.next(bars, is_peer, abort_flag, status);
         rd.template done<kPair>(bars, true);
-        if (tile < 0) break;
-        TileCoord tc;
-        if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-        const int row0 = padded_offsets[tc.expert] + tc.m_block * kRowsPerTile + (int)rank * BM;
+        if (tc.tile < 0) break;
+        const int row0 = tc.poff + tc.m_block * kRowsPerTile + (int)rank * BM;
         const int n0 = tc.n_block * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&bars->done[stage]), phase ^ 1u, abort_flag, status)) { ok = false; break; }
           if (kPair) {
             const uint32_t full = mapa(smem_u32(&bars->full[stage]), 0);
             if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), 2 * (A_STAGE + B_STAGE));
@@ -208,39 +272,41 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-    } else if (warp == 1 && lane == 0 && !is_peer) {
-      // ---------------------------------------------------------------- MMA issuer (leader CTA)
+    } else if ((warp == 1 || warp == 3) && lane == 0 && !is_peer) {
+      // ---------------------------------------------------------------- MMA issuers (leader CTA)
+      // warp 1 owns scratch buffer 0 and the even K blocks (counted across tiles), warp 3 buffer 1 and the odd ones
       constexpr uint32_t idesc = make_idesc_e4m3(kRowsPerTile, BN);
-      int stage = 0; uint32_t phase = 0;
-      int pb = 0; uint32_t pb_phase = 0;
+      const int mine = warp == 1 ? 0 : 1;
+      const uint32_t d_tmem = tmem_base + (uint32_t)(mine * BN);
+      // This thread's K blocks sit two apart, across tile borders: `skip` is 1 when the next tile starts with the
+      // other thread's block.  kStages is even, so the stage index keeps this thread's parity.
+      int stage = mine; uint32_t phase = 0;
+      uint32_t pb_phase = 0;
+      int skip = mine;
       bool ok = true;
       Ring rd;
       for (; ok;) {
-        const int tile = rd.next(bars, false, abort_flag, status);
+        const TileInfo tc = rd.next(bars, false, abort_flag, status);
         rd.template done<kPair>(bars, true);
-        if (tile < 0) break;
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(smem_u32(&bars->part_empty[pb]), pb_phase ^ 1u, abort_flag, status)) { ok = false; break; }
-          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(pb * BN);
+        if (tc.tile < 0) break;
+        int kb = skip;
+        for (; kb < num_kb; kb += 2) {
           const uint64_t adesc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE));
           const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + stage * B_STAGE));
-#pragma unroll
-          for (int k4 = 0; k4 < BKB / 32; ++k4) {        // 32 e4m3 elements of K per MMA
-            if (kPair) tc_mma_f8_pair(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, k4 != 0 ? 1u : 0u);
-            else tc_mma_f8(d_tmem, adesc + (uint64_t)(k4 * 2), bdesc + (uint64_t)(k4 * 2), idesc, k4 != 0 ? 1u : 0u);
-          }
-          if (kPair) {
-            tc_commit_pair_both(smem_u32(&bars->empty[stage]), 3);
-            tc_commit_pair_both(smem_u32(&bars->part_full[pb]), 3);
-          } else {
-            tc_commit(smem_u32(&bars->empty[stage]));
-            tc_commit(smem_u32(&bars->part_full[pb]));
-          }
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
+          // both tests are in flight together; the operands have normally landed long before the buffer is free
+          const bool have_ops = mbar_try_wait(smem_u32(&bars->full[stage]), phase);
+          const bool have_buf = mbar_try_wait(smem_u32(&bars->part_empty[mine]), pb_phase ^ 1u);
+          if (!have_ops && !mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status)) { ok = false; break; }
+          if (!have_buf && !mbar_wait(smem_u32(&bars->part_empty[mine]), pb_phase ^ 1u, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          issue_k_block<kPair>(d_tmem, adesc, bdesc, idesc);
+          if (kPair) tc_commit_pair_both(smem_u32(&bars->done[stage]), 3);
+          else tc_commit(smem_u32(&bars->done[stage]));
+          pb_phase ^= 1u;
+          stage += 2;
+          if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
         }
+        skip = kb - num_kb;                              // 0 or 1
       }
     } else if (warp == 2 && lane == 0 && !is_peer) {
       // ---------------------------------------------------------------- tile scheduler (leader CTA)
@@ -249,8 +315,19 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1u, abort_flag, status)) break;
         int t = atomicAdd(tile_counter, 1);
         if (t >= total_tiles) t = -1;
-        bars->sched_tile[slot] = t;
-        if (kPair) st_shared_cluster_u32(mapa(smem_u32(&bars->sched_tile[slot]), 1), (uint32_t)t);
+        int f[6] = {t, 0, 0, 0, 0, 0};
+        TileCoord tc;
+        if (t >= 0 && decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, t, &tc)) {
+          f[1] = tc.expert; f[2] = tc.m_block; f[3] = tc.n_block;
+          f[4] = counts[tc.expert]; f[5] = padded_offsets[tc.expert];
+        } else {
+          f[0] = t = -1;
+        }
+#pragma unroll
+        for (int i = 5; i >= 0; --i) {                   // the tile id, which readers test for poison, goes last
+          bars->sched_tile[slot][i] = f[i];
+          if (kPair) st_shared_cluster_u32(mapa(smem_u32(&bars->sched_tile[slot][i]), 1), (uint32_t)f[i]);
+        }
         mbar_arrive(smem_u32(&bars->sched_full[slot]));
         if (kPair) mbar_arrive_release_cluster(mapa(smem_u32(&bars->sched_full[slot]), 1));
         if (t < 0) break;
@@ -263,24 +340,28 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
     const int pw = warp - kPromoWarp0;                 // 0..7
     const int lane_grp = warp & 3;                     // tensor-memory lanes 32*lane_grp..+31
     const int half = pw >> 2;                          // which 2x64 columns of the tile
+    uint8_t* my_store = s_store + pw * kStoreStage;
     // column groups: swiglu tile = [128 gate | 128 up] -> this thread owns gate cols 64*half..+63 and the
     // matching up cols; plain tile -> cols 128*half..+127 (two groups of 64 under one weight-scale block)
     const int col0 = kSwiglu ? 64 * half : 128 * half;
     const int col1 = kSwiglu ? 128 + 64 * half : 128 * half + 64;
-    int pb = 0; uint32_t pb_phase = 0;
+    int stage = 0; uint32_t phase = 0;                 // K blocks are consumed in order; buffer = stage parity
+    const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+    // where the "buffer read out" arrivals go: the leader CTA's barriers
+    const uint32_t part_empty0 = kPair ? mapa(smem_u32(&bars->part_empty[0]), 0) : smem_u32(&bars->part_empty[0]);
+    const uint32_t part_empty1 = kPair ? mapa(smem_u32(&bars->part_empty[1]), 0) : smem_u32(&bars->part_empty[1]);
     uint32_t tile_parity = 0;
     Ring rd;
     unsigned long long acc2[64];                       // 128 fp32 accumulators as packed pairs
     for (;;) {
-      const int tile = rd.next(bars, is_peer, abort_flag, status);
+      const TileInfo tc = rd.next(bars, is_peer, abort_flag, status);
       __syncwarp();
       rd.template done<kPair>(bars, lane == 0);
-      if (tile < 0) break;
-      TileCoord tc;
-      if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
-      const int r_in_group = tc.m_block * kRowsPerTile + (int)rank * BM + lane_grp * 32 + lane;
-      const bool row_ok = r_in_group < counts[tc.expert];
-      const size_t grow = (size_t)(padded_offsets[tc.expert] + r_in_group);
+      if (tc.tile < 0) break;
+      const int r_warp = tc.m_block * kRowsPerTile + (int)rank * BM + lane_grp * 32;   // first row of this warp in the group
+      const int r_in_group = r_warp + lane;
+      const bool row_ok = r_in_group < tc.count;
+      const size_t grow = (size_t)(tc.poff + r_in_group);
       const float* sa_row = a_scales + grow * num_kb;
       const int nb0 = 2 * tc.n_block + (kSwiglu ? 0 : half), nb1 = kSwiglu ? nb0 + 1 : nb0;
       const float* sw0_p = b_scales + ((size_t)tc.expert * (2 * n_blocks_n) + nb0) * num_kb;
@@ -288,9 +369,10 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
 #pragma unroll
       for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
       bool ok = true;
-      // Software-pipelined promotion: the partial tile is read in four 32-column chunks per K block; the
-      // load of chunk i+1 is in flight while chunk i is multiplied and added, across K-block borders, and
-      // the scratch buffer is handed back to the MMA warp as soon as its last chunk has been read.
+      // Promotion of one K block: its scratch buffer is read in four 32-column chunks through two staging arrays.
+      // The first two chunks are requested together the moment the block's MMAs have completed, the other two as
+      // the staging arrays drain, and the buffer goes back to its MMA thread as soon as the fourth chunk sits in
+      // registers: the time a buffer stays with these warps is on the critical loop MMA -> promotion -> MMA.
 #define CEP_FMA_CHUNK(V, BASE, S)                                                                   \
   {                                                                                                  \
     const unsigned long long s2_ = pack_f32x2(__float_as_uint(S), __float_as_uint(S));              \
@@ -299,10 +381,12 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   }
       uint32_t va[32], vb[32];
       {
-        const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);
+        const bool got = mbar_wait(smem_u32(&bars->done[stage]), phase, abort_flag, status);
         if (!__all_sync(0xffffffffu, got)) break;
         tc_fence_after();
-        tc_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN + col0), va);
+        const uint32_t t_addr = t_lane + (uint32_t)((stage & 1) * BN);
+        tc_ld32(t_addr + (uint32_t)col0, va);
+        tc_ld32(t_addr + (uint32_t)(col0 + 32), vb);
         tc_wait_ld();
       }
       // the scales of K block kb+1 are fetched while block kb is promoted: their L2 latency would otherwise sit
@@ -310,38 +394,44 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
       float sa_n = row_ok ? __ldg(sa_row) : 0.f, sw0_n = __ldg(sw0_p), sw1_n = __ldg(sw1_p);
       for (int kb = 0; kb < num_kb; ++kb) {
         const float s0 = sa_n * sw0_n, s1 = sa_n * sw1_n;
-        if (kb + 1 < num_kb) {
+        const bool more = kb + 1 < num_kb;
+        if (more) {
           sa_n = row_ok ? __ldg(sa_row + kb + 1) : 0.f;
           sw0_n = __ldg(sw0_p + kb + 1);
           sw1_n = __ldg(sw1_p + kb + 1);
         }
-        const uint32_t t_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN);
-        tc_ld32(t_addr + (uint32_t)(col0 + 32), vb);
+        const int pb = stage & 1;
+        const uint32_t t_addr = t_lane + (uint32_t)(pb * BN);
+        int nstage = stage + 1; uint32_t nphase = phase;
+        if (nstage == kStages) { nstage = 0; nphase ^= 1u; }
         CEP_FMA_CHUNK(va, 0, s0);
-        tc_wait_ld();
         tc_ld32(t_addr + (uint32_t)col1, va);
         CEP_FMA_CHUNK(vb, 16, s0);
-        tc_wait_ld();
         tc_ld32(t_addr + (uint32_t)(col1 + 32), vb);
-        CEP_FMA_CHUNK(va, 32, s1);
+        // the next K block's barrier is tested now: the test's latency hides behind the loads
+        const bool next_ready = more ? mbar_try_wait(smem_u32(&bars->done[nstage]), nphase) : true;
         tc_wait_ld();
         // every column of this scratch buffer is in registers: give it back
         tc_fence_before();
         __syncwarp();
         if (lane == 0) {
-          if (kPair) mbar_arrive_cluster(mapa(smem_u32(&bars->part_empty[pb]), 0));
-          else mbar_arrive(smem_u32(&bars->part_empty[pb]));
+          if (kPair) mbar_arrive_cluster(pb ? part_empty1 : part_empty0);
+          else mbar_arrive(pb ? part_empty1 : part_empty0);
         }
-        if (++pb == 2) { pb = 0; pb_phase ^= 1u; }
-        if (kb + 1 < num_kb) {
-          const bool got = mbar_wait(smem_u32(&bars->part_full[pb]), pb_phase, abort_flag, status);
-          if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+        stage = nstage; phase = nphase;
+        CEP_FMA_CHUNK(va, 32, s1);
+        if (more) {
+          if (!__all_sync(0xffffffffu, next_ready)) {
+            const bool got = mbar_wait(smem_u32(&bars->done[stage]), phase, abort_flag, status);
+            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+          }
           tc_fence_after();
-          tc_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(pb * BN + col0), va);
-          CEP_FMA_CHUNK(vb, 48, s1);
+          tc_ld32(t_lane + (uint32_t)((stage & 1) * BN + col0), va);
+        }
+        CEP_FMA_CHUNK(vb, 48, s1);
+        if (more) {
+          tc_ld32(t_lane + (uint32_t)((stage & 1) * BN + col0 + 32), vb);
           tc_wait_ld();
-        } else {
-          CEP_FMA_CHUNK(vb, 48, s1);
         }
       }
 #undef CEP_FMA_CHUNK
@@ -371,37 +461,40 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
         amax = fmaxf(amax, *theirs);
         tile_parity ^= 1u;
         const float scale = amax == 0.f ? 1.f : __fdiv_rn(amax, 448.f);
-        if (row_ok) {
-          uint4* dst = reinterpret_cast<uint4*>(out_codes + grow * out_ld + tc.n_block * 128 + 64 * half);
+        const float inv = __fdiv_rn(1.f, scale);         // one division per row; the 64 quotients become products
+        // 64 codes per row: through the warp's staging buffer, so that a store instruction covers 64 contiguous
+        // bytes of 8 rows instead of 16 bytes of 32 rows
+        uint4 ch[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int i = q * 16 + j * 4;
+            const uint32_t lo = cvt_e4m3x2(acc[i] * inv, acc[i + 1] * inv);
+            const uint32_t hi = cvt_e4m3x2(acc[i + 2] * inv, acc[i + 3] * inv);
+            w[j] = lo | (hi << 16);
+          }
+          ch[q] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        store_rows_64B(my_store, lane, ch, out_codes + (size_t)(tc.poff + r_warp) * out_ld + tc.n_block * 128 + 64 * half,
+                       (size_t)out_ld, tc.count - r_warp);
+        if (half == 0 && row_ok) out_scales[grow * (n_out_cols / 128) + tc.n_block] = scale;
+      } else {
+        // 128 bf16 per row, 32 columns (64 bytes) per pass through the staging buffer
+        uint8_t* orow = reinterpret_cast<uint8_t*>(out_bf16 + (size_t)(tc.poff + r_warp) * out_ld + tc.n_block * BN + 128 * half);
+#pragma unroll
+        for (int pass = 0; pass < 4; ++pass) {
+          uint4 ch[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int i = q * 16 + j * 4;
-              const uint32_t lo = cvt_e4m3x2(__fdiv_rn(acc[i], scale), __fdiv_rn(acc[i + 1], scale));
-              const uint32_t hi = cvt_e4m3x2(__fdiv_rn(acc[i + 2], scale), __fdiv_rn(acc[i + 3], scale));
-              w[j] = lo | (hi << 16);
-            }
-            dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            const int i = 32 * pass + 8 * q;
+            ch[q].x = pack_bf16(acc[i + 0], acc[i + 1]);
+            ch[q].y = pack_bf16(acc[i + 2], acc[i + 3]);
+            ch[q].z = pack_bf16(acc[i + 4], acc[i + 5]);
+            ch[q].w = pack_bf16(acc[i + 6], acc[i + 7]);
           }
-          if (half == 0) out_scales[grow * (n_out_cols / 128) + tc.n_block] = scale;
-        }
-      } else {
-        if (row_ok) {
-          const int c_out = tc.n_block * BN + 128 * half;
-          if (c_out < n_out_cols) {
-            uint4* dst = reinterpret_cast<uint4*>(out_bf16 + grow * out_ld + c_out);
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              uint4 v;
-              v.x = pack_bf16(acc[8 * q + 0], acc[8 * q + 1]);
-              v.y = pack_bf16(acc[8 * q + 2], acc[8 * q + 3]);
-              v.z = pack_bf16(acc[8 * q + 4], acc[8 * q + 5]);
-              v.w = pack_bf16(acc[8 * q + 6], acc[8 * q + 7]);
-              dst[q] = v;
-            }
-          }
+          store_rows_64B(my_store, lane, ch, orow + 64 * pass, (size_t)out_ld * 2, tc.count - r_warp);
         }
       }
     }
@@ -437,8 +530,10 @@ __global__ void pack_scales_kernel(const float* __restrict__ s_gate, const float
   }
 }
 
-int g_clusters = -1;
-bool g_single_ready = false;
+// cudaFuncSetAttribute and the occupancy answer hold per device: one slot per device ordinal
+constexpr int kMaxDevices = 64;
+int g_clusters[kMaxDevices];                           // co-resident CTA pairs + 1 (0: not set up yet)
+bool g_single_ready[kMaxDevices];
 
 template <bool kPair>
 cudaError_t set_smem_attr() {
@@ -449,8 +544,8 @@ cudaError_t set_smem_attr() {
                               Geo<kPair>::kSmemBytes);
 }
 
-cudaError_t setup_pair(int n_sms) {
-  if (g_clusters >= 0) return cudaSuccess;
+cudaError_t setup_pair(int dev, int n_sms) {
+  if (g_clusters[dev] > 0) return cudaSuccess;
   cudaError_t e = set_smem_attr<true>();
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -462,11 +557,13 @@ cudaError_t setup_pair(int n_sms) {
   int n = 0;
   e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_fp8_kernel<true, true>, &cfg);
   if (e != cudaSuccess) return e;
-  g_clusters = n;
+  g_clusters[dev] = n + 1;
   return cudaSuccess;
 }
 
 }  // namespace
+
+int gemm_fp8_box_rows(int pair) { return pair ? BN / 2 : BN; }
 
 cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const float* s_up, const float* s_down,
                                float* s13p, float* s2p, cudaStream_t s, int64_t* launches) {
@@ -487,23 +584,27 @@ static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, con
                             counter, lp.status);
 }
 
-// pair != 0: CTA pairs on 256x256 tiles (the weight operand map must have a 128-row box, max_tiles counts pair
-// tiles); pair == 0: one CTA per 128x256 tile (256-row box, max_tiles counts single tiles).
+// pair != 0: CTA pairs on 256x256 tiles, max_tiles counts pair tiles; pair == 0: one CTA per 128x256 tile,
+// max_tiles counts single tiles.  The weight operand map must have a box of gemm_fp8_box_rows(pair) rows.
 cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                             const float* a_scales, const float* b_scales, void* out, float* out_scales,
                             const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches) {
-  cudaError_t e;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   int ctas;
   if (pair) {
-    e = setup_pair(n_sms);
+    e = setup_pair(dev, n_sms);
     if (e != cudaSuccess) return e;
-    if (g_clusters < 1) return cudaErrorNotSupported;
-    ctas = 2 * (max_tiles < g_clusters ? max_tiles : g_clusters);
+    const int clusters = g_clusters[dev] - 1;
+    if (clusters < 1) return cudaErrorNotSupported;
+    ctas = 2 * (max_tiles < clusters ? max_tiles : clusters);
   } else {
-    if (!g_single_ready) {
+    if (!g_single_ready[dev]) {
       e = set_smem_attr<false>();
       if (e != cudaSuccess) return e;
-      g_single_ready = true;
+      g_single_ready[dev] = true;
     }
     ctas = max_tiles < n_sms ? max_tiles : n_sms;
   }

@@ -428,7 +428,8 @@ int moe_load_weights(cep_plan* p, const void* w_gate, const void* w_up, const vo
   if (c.gemm_impl != CEP_GEMM_SIMT) {
     const int elt = fp8 ? 1 : 2;
     // the CTA-pair kernel loads half a weight tile per CTA
-    const int box = c.gemm_impl == CEP_GEMM_TCGEN05 ? gemm_tile_cols() / 2 : gemm_tile_cols();
+    const int box = fp8 ? gemm_fp8_box_rows(c.gemm_impl == CEP_GEMM_TCGEN05)
+                        : c.gemm_impl == CEP_GEMM_TCGEN05 ? gemm_tile_cols() / 2 : gemm_tile_cols();
     int r1 = make_operand_map(&p->tm_b1, p->w13p, elt, c.hidden, 2 * c.inter, c.n_experts_local, box);
     int r2 = make_operand_map(&p->tm_b2, p->w2p, elt, c.inter, c.hidden, c.n_experts_local, box);
     if (r1 || r2) return fail(p, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the weight operands failed (%d, %d)", r1, r2);
