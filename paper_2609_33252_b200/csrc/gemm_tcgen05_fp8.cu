@@ -369,30 +369,30 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
 #pragma unroll
       for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
       bool ok = true;
-      // Promotion of one K block: its scratch buffer is read in four 32-column chunks through two staging arrays.
-      // The first two chunks are requested together the moment the block's MMAs have completed, the other two as
-      // the staging arrays drain, and the buffer goes back to its MMA thread as soon as the fourth chunk sits in
-      // registers: the time a buffer stays with these warps is on the critical loop MMA -> promotion -> MMA.
-#define CEP_FMA_CHUNK(V, BASE, S)                                                                   \
+      // Promotion of one K block.  How long a scratch buffer stays with these warps is on the critical loop
+      // MMA -> promotion -> MMA, so nothing but the reads themselves sits between "the block's MMAs have completed"
+      // and "buffer handed back": this thread's 128 values are read in two 64-column loads, and only the first
+      // half's multiply-adds (which free the staging registers for the second load) run in between.
+#define CEP_FMA_HALF(BASE, S)                                                                       \
   {                                                                                                  \
     const unsigned long long s2_ = pack_f32x2(__float_as_uint(S), __float_as_uint(S));              \
-    _Pragma("unroll") for (int i = 0; i < 16; ++i)                                                  \
-        fma_f32x2(acc2[(BASE) + i], pack_f32x2((V)[2 * i], (V)[2 * i + 1]), s2_);                  \
+    _Pragma("unroll") for (int i = 0; i < 32; ++i)                                                  \
+        fma_f32x2(acc2[(BASE) + i], pack_f32x2(v[2 * i], v[2 * i + 1]), s2_);                      \
   }
-      uint32_t va[32], vb[32];
-      {
-        const bool got = mbar_wait(smem_u32(&bars->done[stage]), phase, abort_flag, status);
-        if (!__all_sync(0xffffffffu, got)) break;
-        tc_fence_after();
-        const uint32_t t_addr = t_lane + (uint32_t)((stage & 1) * BN);
-        tc_ld32(t_addr + (uint32_t)col0, va);
-        tc_ld32(t_addr + (uint32_t)(col0 + 32), vb);
-        tc_wait_ld();
-      }
+      uint32_t v[64];
       // the scales of K block kb+1 are fetched while block kb is promoted: their L2 latency would otherwise sit
       // in front of every block's first multiply-add
       float sa_n = row_ok ? __ldg(sa_row) : 0.f, sw0_n = __ldg(sw0_p), sw1_n = __ldg(sw1_p);
+      bool ready = false;                                // outcome of the early test of this K block's barrier
       for (int kb = 0; kb < num_kb; ++kb) {
+        if (!__all_sync(0xffffffffu, ready)) {
+          const bool got = mbar_wait(smem_u32(&bars->done[stage]), phase, abort_flag, status);
+          if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+        }
+        tc_fence_after();
+        const int pb = stage & 1;
+        const uint32_t t_addr = t_lane + (uint32_t)(pb * BN);
+        tc_ld64(t_addr + (uint32_t)col0, v);
         const float s0 = sa_n * sw0_n, s1 = sa_n * sw1_n;
         const bool more = kb + 1 < num_kb;
         if (more) {
@@ -400,16 +400,10 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           sw0_n = __ldg(sw0_p + kb + 1);
           sw1_n = __ldg(sw1_p + kb + 1);
         }
-        const int pb = stage & 1;
-        const uint32_t t_addr = t_lane + (uint32_t)(pb * BN);
-        int nstage = stage + 1; uint32_t nphase = phase;
-        if (nstage == kStages) { nstage = 0; nphase ^= 1u; }
-        CEP_FMA_CHUNK(va, 0, s0);
-        tc_ld32(t_addr + (uint32_t)col1, va);
-        CEP_FMA_CHUNK(vb, 16, s0);
-        tc_ld32(t_addr + (uint32_t)(col1 + 32), vb);
-        // the next K block's barrier is tested now: the test's latency hides behind the loads
-        const bool next_ready = more ? mbar_try_wait(smem_u32(&bars->done[nstage]), nphase) : true;
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        tc_wait_ld();
+        CEP_FMA_HALF(0, s0);
+        tc_ld64(t_addr + (uint32_t)col1, v);
         tc_wait_ld();
         // every column of this scratch buffer is in registers: give it back
         tc_fence_before();
@@ -418,23 +412,11 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           if (kPair) mbar_arrive_cluster(pb ? part_empty1 : part_empty0);
           else mbar_arrive(pb ? part_empty1 : part_empty0);
         }
-        stage = nstage; phase = nphase;
-        CEP_FMA_CHUNK(va, 32, s1);
-        if (more) {
-          if (!__all_sync(0xffffffffu, next_ready)) {
-            const bool got = mbar_wait(smem_u32(&bars->done[stage]), phase, abort_flag, status);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-          }
-          tc_fence_after();
-          tc_ld32(t_lane + (uint32_t)((stage & 1) * BN + col0), va);
-        }
-        CEP_FMA_CHUNK(vb, 48, s1);
-        if (more) {
-          tc_ld32(t_lane + (uint32_t)((stage & 1) * BN + col0 + 32), vb);
-          tc_wait_ld();
-        }
+        // the next K block's barrier is tested now: the test's latency hides behind the second half's arithmetic
+        ready = more ? mbar_try_wait(smem_u32(&bars->done[stage]), phase) : false;
+        CEP_FMA_HALF(32, s1);
       }
-#undef CEP_FMA_CHUNK
+#undef CEP_FMA_HALF
       if (!ok) break;
       // ---------------------------------------------------------------- epilogue from registers
       float acc[128];
