@@ -61,7 +61,8 @@ typedef enum {
   CEP_ERR_CAPACITY = -4,       /* more tokens or chunks than the plan was made for              */
   CEP_ERR_INCOMPLETE = -5,     /* flush/combine with fewer chunks than ffn_begin announced;
                                   the work already submitted still runs                          */
-  CEP_ERR_BAD_ROUTING = -6,    /* device found an expert id outside [0, n_experts_global)       */
+  CEP_ERR_BAD_ROUTING = -6,    /* device found an expert id outside [0, n_experts_global), or (plans
+                                  made with debug_checks) a token naming one expert twice        */
   CEP_ERR_DEVICE_TIMEOUT = -7, /* a bounded wait inside a kernel expired; kernel exited cleanly */
   CEP_ERR_CUDA = -8,           /* a CUDA runtime/driver call failed                             */
   CEP_ERR_UNSUPPORTED = -9     /* valid request this build does not implement                   */
@@ -71,7 +72,7 @@ typedef enum {
   CEP_BF16 = 0,                /* bf16 activations and weights, fp32 accumulate, bf16 output    */
   CEP_FP8_E4M3_BLOCK128 = 1,   /* e4m3 codes; fp32 scales per 1x128 activation block and per
                                   128x128 weight block; bf16 output                              */
-  CEP_MXFP4_E4M3 = 2           /* microscaling: MXFP4 expert weights (Section 5.1), e2m1 codes with
+  CEP_MXFP4_E4M3 = 2           /* microscaling: MXFP4 expert weights ("Evaluation Settings"), e2m1 codes with
                                   one ue8m0 scale (2^(s-127)) per 32 elements of the input
                                   dimension; e4m3 activations with one ue8m0 scale per 1x32 block
                                   along the hidden dimension; the intermediate is re-quantised the
@@ -80,7 +81,7 @@ typedef enum {
                                   fp32 accumulate; bf16 output                                   */
 } cep_dtype;
 
-/* Execution modes of the ablation in Section 5.4. */
+/* Execution modes of the ablation study ("Deep Dive"). */
 typedef enum {
   CEP_MODE_SYNC = 0,           /* one invocation once all chunks have arrived                   */
   CEP_MODE_ASYNC = 1,          /* one invocation per chunk as it arrives                        */
@@ -112,9 +113,11 @@ typedef struct {
   int32_t gemm_impl;           /* cep_gemm_impl                                                 */
   int32_t debug_checks;        /* nonzero: every region of the workspace is followed by a 1 KiB gap
                                   filled with a byte pattern at moe_plan (cep_debug_check_guards
-                                  verifies them).  The in-kernel checks (expert ids in range, rows
-                                  inside the scratch slot, tile-ring values) are always on and
-                                  record in the status word instead of trapping                 */
+                                  verifies them), and the histogram kernel also checks that the
+                                  top_k ids of a token are distinct (CEP_ERR_BAD_ROUTING).  The
+                                  other in-kernel checks (expert ids in range, rows inside the
+                                  scratch slot, tile-ring values) are always on and record in the
+                                  status word instead of trapping                               */
   int32_t profile_kernels;     /* nonzero: record CUDA events between the kernels of every
                                   invocation so ffn_query can report per-kernel device times    */
   int32_t reserved_;           /* set to 0                                                      */
@@ -167,10 +170,12 @@ CEP_API int moe_load_weights(cep_plan* plan, const void* w_gate, const void* w_u
                      void* packed, size_t packed_bytes, void* stream);
 
 /*
- * Open a layer call.  `out` [device] bf16 [n_tokens_total, H] in token order; every row
- * is written by combine work (rows of tokens with no local expert become exact zeros).
- * n_chunks_expected chunks will be submitted, together covering the n_tokens_total
- * tokens exactly once.
+ * Open a layer call.  `out` [device] bf16 [n_tokens_total, H] in token order, 16-byte aligned
+ * (CEP_ERR_ARG otherwise); every row is written by combine work (rows of tokens with no local
+ * expert become exact zeros).  n_chunks_expected chunks will be submitted, together covering the
+ * n_tokens_total tokens exactly once: a chunk that would bring the submitted tokens above
+ * n_tokens_total is refused with CEP_ERR_CAPACITY, and a flush or combine with all chunks in but
+ * fewer tokens than announced reports CEP_ERR_INCOMPLETE.
  */
 CEP_API int ffn_begin(cep_plan* plan, void* out, int32_t n_tokens_total, int32_t n_chunks_expected);
 
@@ -227,7 +232,8 @@ CEP_API int combine(cep_plan* plan, void* stream);
 
 /* Device-side status of the last closed layer call.  Valid after the stream given to
  * combine() has completed (the caller synchronises); before that returns CEP_ERR_STATE.
- * CEP_OK, CEP_ERR_BAD_ROUTING or CEP_ERR_DEVICE_TIMEOUT. */
+ * CEP_OK, CEP_ERR_BAD_ROUTING, CEP_ERR_DEVICE_TIMEOUT, or CEP_ERR_CAPACITY (a row index left
+ * the scratch slot: more local pairs than the plan was made for; the access was skipped). */
 CEP_API int ffn_status(cep_plan* plan);
 
 /*
@@ -283,8 +289,8 @@ typedef struct {
 } cep_calibration;
 
 /*
- * Launch-threshold calibration (Section 3.2: theta is "the smallest profiled count that reaches at least rho of
- * the observed peak FFN throughput"; Section 4.2 models FFN latency from the same profile).  Runs the plan's OWN
+ * Launch-threshold calibration (Section 3.2: theta is the smallest profiled expert-token count whose FFN throughput
+ * reaches the fraction rho of the best profiled one; Section 3.3, Eq. 2 models FFN latency from the same profile).  Runs the plan's OWN
  * kernels, with the weights it holds, on synthetic routing that gives every local expert rows_per_expert[i] rows
  * (ascending), `reps` timed layer calls per point after two warm-ups, and then probes how many compute streams a
  * chain of theta-sized invocations wants.  Blocks the host until done; not part of the hot path.  Needs a plan
@@ -329,8 +335,10 @@ CEP_API const char* cep_last_error(const cep_plan* plan);
  *                   [1] != 0 a row did not fit pair_of_row_capacity
  * Limits: n_experts_local <= 1024 and ceil(n_tokens*top_k / 2048) * n_experts_local <= 262144;
  * larger requests return CEP_ERR_CAPACITY.  The work is enqueued on `stream`; outputs are ready when
- * it completes.  The first call on each device looks up the array's device address (a blocking
- * runtime query), so make that first call before any stream capture.  All calls share the one array,
+ * it completes.  The first call on each device looks up the array's device address: a blocking
+ * runtime query that also loads the library's device code onto that GPU if nothing has yet, so make
+ * that first call once at start-up, before any stream capture and off any latency-critical path.
+ * All calls share the one array,
  * which keeps the previous call's contents (the part that must start at zero is cleared by every
  * call): calls whose GPU work may overlap must be ordered by the caller or they race.
  */

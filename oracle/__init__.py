@@ -13,7 +13,7 @@ Contents (each function cites the passage of the paper it restates):
 * ``schedule``         streamFFN launch decisions: threshold batching, final flush, the
                        Sync / Async / Async+streamFFN modes, round-robin streams
                        (Section 3.2 "Launch threshold", "Multi-stream execution";
-                       Section 5.4 ablation modes)
+                       "Deep Dive", ablation study: the three modes)
 * ``moe_forward``      the fp64 layer result (C, ``oracle_moe.c``)
 * codecs               bf16 / e4m3 / e2m1 / ue8m0 decode and encode, the microscaling block
                        scale rule (C)
@@ -34,7 +34,7 @@ _SO = os.path.join(_HERE, "liboracle_moe.so")
 _SRC = os.path.join(_HERE, "oracle_moe.c")
 
 F64, BF16, FP8, MXFP4 = 0, 1, 2, 3
-MIRROR_FP8_ACT, MIRROR_BF16_ACT, MIRROR_MXFP8_ACT = 1, 2, 4
+MIRROR_FP8_ACT, MIRROR_MXFP8_ACT = 1, 4
 
 
 def build(force: bool = False) -> str:

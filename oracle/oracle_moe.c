@@ -21,7 +21,7 @@
  * and loop nest, dense-MLP special cases through library matmuls, closed forms of
  * silu, exhaustive codec tables.  No function here is "parity unpinned".
  *
- * Microscaling operands (Section 5.1: the routed-expert weights of two of the three
+ * Microscaling operands ("Evaluation Settings", models and environments: the routed-expert weights of two of the three
  * evaluated models are MXFP4): a block of 32 consecutive elements along the contraction
  * dimension shares one power-of-two scale stored as an 8-bit exponent (ue8m0); weights are
  * e2m1 elements, activations e4m3 elements.  The paper gives no quantisation rule; the one
@@ -37,7 +37,7 @@
 #endif
 
 enum { ORACLE_F64 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2, ORACLE_MXFP4 = 3 };
-enum { ORACLE_MIRROR_FP8_ACT = 1, ORACLE_MIRROR_BF16_ACT = 2, ORACLE_MIRROR_MXFP8_ACT = 4 };
+enum { ORACLE_MIRROR_FP8_ACT = 1, ORACLE_MIRROR_MXFP8_ACT = 4 };
 
 /* ---- codecs: exact decoders and the two round-to-nearest-even encoders ---- */
 
@@ -269,8 +269,6 @@ int oracle_moe_forward(int dtype, int64_t T, int64_t H, int64_t I, int64_t E_loc
         for (int64_t i = 0; i < I; ++i) g[i] = oracle_silu(g[i]) * u[i];   /* a = silu(g) * u */
         if (mirror & ORACLE_MIRROR_FP8_ACT) requant_fp8_row(g, I);
         if (mirror & ORACLE_MIRROR_MXFP8_ACT) requant_mxfp8_row(g, I);
-        if (mirror & ORACLE_MIRROR_BF16_ACT)
-          for (int64_t i = 0; i < I; ++i) g[i] = oracle_bf16_to_f64(oracle_f64_to_bf16(g[i]));
         for (int64_t h = 0; h < H; ++h) y[h] = 0.0;
         for (int64_t i = 0; i < I; ++i) {         /* i ascending for every h */
           double av = g[i];

@@ -498,10 +498,19 @@ int make_operand_map(GemmTensorMap* out, const void* base, int elt_bytes, int K,
 int gemm_tile_rows() { return BM; }
 int gemm_tile_cols() { return BN; }
 
-static int g_pair_clusters = -1;      // co-resident CTA pairs on this device (0: pairs unavailable)
+// cudaFuncSetAttribute and the occupancy answer hold per device: one slot per device ordinal
+constexpr int kMaxDevices = 64;
+static int g_pair_clusters[kMaxDevices];   // co-resident CTA pairs on the device + 1 (0: not set up yet)
+static bool g_single_ready[kMaxDevices];
 
-static cudaError_t setup_pair_kernels(int n_sms) {
-  if (g_pair_clusters >= 0) return cudaSuccess;
+static cudaError_t current_device(int* dev) {
+  cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return e;
+  return (*dev < 0 || *dev >= kMaxDevices) ? cudaErrorInvalidDevice : cudaSuccess;
+}
+
+static cudaError_t setup_pair_kernels(int dev, int n_sms) {
+  if (g_pair_clusters[dev] > 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
@@ -515,22 +524,24 @@ static cudaError_t setup_pair_kernels(int n_sms) {
   int n = 0;
   e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_bf16_pair_kernel<true>, &cfg);
   if (e != cudaSuccess) return e;
-  g_pair_clusters = n;
+  g_pair_clusters[dev] = n + 1;
   return cudaSuccess;
 }
-
-int gemm_pair_clusters() { return g_pair_clusters; }
 
 cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                                      void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
                                      int64_t* launches) {
   if (p.is_fp8) return cudaErrorNotSupported;
-  cudaError_t e = setup_pair_kernels(n_sms);
+  int dev = 0;
+  cudaError_t e = current_device(&dev);
   if (e != cudaSuccess) return e;
-  if (g_pair_clusters < 1) return cudaErrorNotSupported;
+  e = setup_pair_kernels(dev, n_sms);
+  if (e != cudaSuccess) return e;
+  const int resident = g_pair_clusters[dev] - 1;
+  if (resident < 1) return cudaErrorNotSupported;
   const int n_blocks_n = (p.N + BN - 1) / BN;
   const int n_out_cols = p.swiglu ? p.N / 2 : p.N;
-  int clusters = max_pair_tiles < g_pair_clusters ? max_pair_tiles : g_pair_clusters;
+  int clusters = max_pair_tiles < resident ? max_pair_tiles : resident;
   if (clusters < 1) return cudaSuccess;
   int num_kb = p.K * 2 / BKB;
   int n_experts = p.n_experts, out_ld = p.out_ld;
@@ -561,13 +572,15 @@ cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a,
                                 void* out, const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s,
                                 int64_t* launches) {
   if (p.is_fp8) return cudaErrorNotSupported;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(grouped_gemm_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  int dev = 0;
+  cudaError_t e = current_device(&dev);
+  if (e != cudaSuccess) return e;
+  if (!g_single_ready[dev]) {
+    e = cudaFuncSetAttribute(grouped_gemm_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(grouped_gemm_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    g_single_ready[dev] = true;
   }
   const int n_blocks_n = (p.N + BN - 1) / BN;
   const int n_out_cols = p.swiglu ? p.N / 2 : p.N;

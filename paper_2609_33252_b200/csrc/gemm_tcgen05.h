@@ -26,7 +26,6 @@ cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a,
 cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                                      void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
                                      int64_t* launches);
-int gemm_pair_clusters();
 
 // Block-scaled e4m3 variant.  a_scales [rows, K/128], b_scales [E, N/128, K/128] fp32.  With p.swiglu the output is
 // e4m3 codes [rows, N/2] plus out_scales [rows, N/256]; otherwise bf16 [rows, N].  pair != 0: CTA pairs on 256x256

@@ -428,10 +428,12 @@ __global__ void pack_weight_sf_kernel(const uint8_t* __restrict__ src, uint8_t* 
   }
 }
 
-int g_clusters = -1;
+// cudaFuncSetAttribute and the occupancy answer hold per device: one slot per device ordinal
+constexpr int kMaxDevices = 64;
+int g_clusters[kMaxDevices];                           // co-resident CTA pairs + 1 (0: not set up yet)
 
-cudaError_t setup(int n_sms) {
-  if (g_clusters >= 0) return cudaSuccess;
+cudaError_t setup(int dev, int n_sms) {
+  if (g_clusters[dev] > 0) return cudaSuccess;
   cudaError_t e = cudaSuccess;
 #define CEP_MX_ATTR(SW, G) if (e == cudaSuccess) e = cudaFuncSetAttribute(grouped_gemm_mx_kernel<SW, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   CEP_MX_ATTR(true, 2) CEP_MX_ATTR(true, 3) CEP_MX_ATTR(false, 2) CEP_MX_ATTR(false, 3)
@@ -446,7 +448,7 @@ cudaError_t setup(int n_sms) {
   int n = 0;
   e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_mx_kernel<true, 2>, &cfg);
   if (e != cudaSuccess) return e;
-  g_clusters = n;
+  g_clusters[dev] = n + 1;
   return cudaSuccess;
 }
 
@@ -516,10 +518,15 @@ cudaError_t launch_prepack_mx(const cep_config& cfg, const void* w_gate, const v
 cudaError_t launch_gemm_mx(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
                            const GemmTensorMap& tm_sfa, const GemmTensorMap& tm_sfb, void* out, void* out_sf,
                            const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s, int64_t* launches) {
-  cudaError_t e = setup(n_sms);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (g_clusters < 1) return cudaErrorNotSupported;
-  const int ctas = 2 * (max_pair_tiles < g_clusters ? max_pair_tiles : g_clusters);
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  e = setup(dev, n_sms);
+  if (e != cudaSuccess) return e;
+  const int resident = g_clusters[dev] - 1;
+  if (resident < 1) return cudaErrorNotSupported;
+  const int ctas = 2 * (max_pair_tiles < resident ? max_pair_tiles : resident);
   if (ctas < 2) return cudaSuccess;
   const int n_blocks_n = p.N / BN;
   const int n_out_cols = p.swiglu ? p.N / 2 : p.N;

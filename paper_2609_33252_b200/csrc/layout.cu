@@ -25,8 +25,8 @@ __device__ __forceinline__ int load_pair_id(const BatchDesc& b, int k, int p /*b
 
 // ---- 1. histogram: per segment of kSegPairs pairs, per local expert
 __global__ void __launch_bounds__(kThreads)
-hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global, int32_t* __restrict__ seg_hist,
-            int32_t* __restrict__ status) {
+hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global, int check_duplicates,
+            int32_t* __restrict__ seg_hist, int32_t* __restrict__ status) {
   extern __shared__ int32_t sh[];
   pdl_enter();
   for (int e = threadIdx.x; e < E; e += kThreads) sh[e] = 0;
@@ -49,6 +49,17 @@ hist_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int E_global,
     else if (e < E) atomicAdd(&sh[e], 1);
   }
   if (bad) atomicOr(&status[kStBadRouting], 1);
+  if (check_duplicates) {                         // debug plans only: a token must not name an expert twice
+    bool dup = false;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const int p = p0 + i * kThreads + threadIdx.x;
+      if (p >= p1) continue;
+      const int j = p % k;
+      for (int j2 = 0; j2 < j; ++j2) dup |= load_pair_id(batch, k, p - j + j2) == ids[i];
+    }
+    if (dup) atomicOr(&status[kStBadRouting], 2);
+  }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += kThreads) seg_hist[(size_t)blockIdx.x * E + e] = sh[e];
 }
@@ -241,7 +252,7 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
   if (n_seg < 1) n_seg = 1;
   cudaError_t err;
   err = launch_pdl(hist_kernel, dim3(n_seg), dim3(kThreads), E * sizeof(int32_t), s, 1, batch, k, E, cfg.n_experts_global,
-                   lp.block_base, lp.status);
+                   cfg.debug_checks != 0 ? 1 : 0, lp.block_base, lp.status);
   if (err != cudaSuccess) return err;
   err = launch_pdl(scan_kernel, dim3(1), dim3(1024), 0, s, 1, n_seg, E, lp.block_base, lp.counts, lp.offsets,
                    lp.padded_offsets, lp.tile_prefix, lp.sched);
@@ -328,7 +339,7 @@ extern "C" int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens,
   batch.n_chunks = 1;
   batch.n_tokens = n_tokens;
   const int E = n_experts_local;
-  hist_kernel<<<(int)n_seg, kThreads, E * sizeof(int32_t), st>>>(batch, top_k, E, n_experts_global, seg_hist, st_words);
+  hist_kernel<<<(int)n_seg, kThreads, E * sizeof(int32_t), st>>>(batch, top_k, E, n_experts_global, 0, seg_hist, st_words);
   scan_kernel<<<1, 1024, 0, st>>>((int)n_seg, E, seg_hist, counts, offsets, padded_offsets, tile_prefix, scratch + 1600);
   rank_kernel<<<(int)n_seg, kThreads, kWarps * E * sizeof(int32_t), st>>>(batch, top_k, E, seg_hist, row_of_pair,
                                                                         pair_of_row, pair_of_row_capacity, st_words);

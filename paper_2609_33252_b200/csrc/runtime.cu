@@ -16,7 +16,7 @@ using namespace cep;
 
 namespace {
 
-char g_error[256] = "";
+thread_local char g_error[256] = "";          // last error of a call that had no plan to record it in
 constexpr int kGuardByte = 0xA5;
 constexpr size_t kStatusBlockBytes = 256;        // one status block (kStWords int32) per layer-call parity
 
@@ -202,6 +202,9 @@ int launch_invocation(cep_plan* p) {
   }
   batch.n_chunks = (int)p->pending.size();
   batch.n_tokens = tok;
+  // nothing is launched for a batch the scratch slot was not carved for
+  if (tok > c.max_tokens || ((long long)tok * c.top_k + kSegPairs - 1) / kSegPairs > p->L.n_seg_max)
+    return fail(p, CEP_ERR_CAPACITY, "a batch of %d tokens exceeds the plan's max_tokens = %d", tok, c.max_tokens);
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->weights_evt, 0));
   for (size_t i = 0; i < p->pending.size(); ++i) CUDA_TRY(p, cudaStreamWaitEvent(st, p->ready_evt[first_pos + (int)i], 0));
@@ -443,6 +446,7 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   if (p->layer_open) return fail(p, CEP_ERR_STATE, "ffn_begin while a layer call is open (call combine first)");
   if (!p->have_weights) return fail(p, CEP_ERR_STATE, "ffn_begin before moe_load_weights");
   if (!out || n_tokens_total < 0 || n_chunks_expected < 0) return fail(p, CEP_ERR_ARG, "bad ffn_begin arguments");
+  if (reinterpret_cast<uintptr_t>(out) % 16) return fail(p, CEP_ERR_ARG, "out must be 16-byte aligned");
   if (n_tokens_total > p->cfg.max_tokens) return fail(p, CEP_ERR_CAPACITY, "%d tokens, plan made for %d", n_tokens_total, p->cfg.max_tokens);
   if (n_chunks_expected > p->cfg.max_chunks) return fail(p, CEP_ERR_CAPACITY, "%d chunks, plan made for %d", n_chunks_expected, p->cfg.max_chunks);
   cudaStream_t s0 = p->streams[0];
@@ -473,6 +477,11 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   if (p->chunk_seen[chunk_id]) return fail(p, CEP_ERR_STATE, "chunk %d submitted twice", chunk_id);
   if (n_tokens < 0 || token_offset < 0) return fail(p, CEP_ERR_ARG, "negative n_tokens or token_offset");
   if ((long long)token_offset + n_tokens > p->n_tokens_total) return fail(p, CEP_ERR_CAPACITY, "chunk %d covers tokens beyond n_tokens_total", chunk_id);
+  // chunks cover the layer call's tokens exactly once: together they can never hold more than n_tokens_total
+  // (which also keeps every batch within max_tokens, the size the scratch slots were carved for)
+  if ((long long)p->tokens_submitted + n_tokens > p->n_tokens_total)
+    return fail(p, CEP_ERR_CAPACITY, "chunk %d brings the submitted tokens to %lld, the layer call has %d", chunk_id,
+                (long long)p->tokens_submitted + n_tokens, p->n_tokens_total);
   if (n_tokens > 0 && (!tokens || !topk_ids || !topk_weights)) return fail(p, CEP_ERR_ARG, "a chunk pointer is NULL");
   if (reinterpret_cast<uintptr_t>(tokens) % 16) return fail(p, CEP_ERR_ARG, "chunk tokens must be 16-byte aligned");
   const bool fp8 = dtype_is_bytes(p->cfg.dtype);
@@ -523,6 +532,8 @@ int ffn_flush(cep_plan* p) {
   if (rc) return rc;
   if (p->n_submitted < p->n_chunks_expected)
     return fail(p, CEP_ERR_INCOMPLETE, "flush after %d of %d chunks", p->n_submitted, p->n_chunks_expected);
+  if (p->tokens_submitted < p->n_tokens_total)
+    return fail(p, CEP_ERR_INCOMPLETE, "the chunks cover %d of the layer call's %d tokens", p->tokens_submitted, p->n_tokens_total);
   return CEP_OK;
 }
 
@@ -533,6 +544,8 @@ int combine(cep_plan* p, void* stream) {
   if (!p->flushed) { rc = ffn_flush(p); if (rc && rc != CEP_ERR_INCOMPLETE) return rc; }
   else if (p->n_submitted < p->n_chunks_expected)
     rc = fail(p, CEP_ERR_INCOMPLETE, "combine after %d of %d chunks", p->n_submitted, p->n_chunks_expected);
+  else if (p->tokens_submitted < p->n_tokens_total)
+    rc = fail(p, CEP_ERR_INCOMPLETE, "the chunks cover %d of the layer call's %d tokens", p->tokens_submitted, p->n_tokens_total);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
   for (const Invocation& iv : p->inv) CUDA_TRY(p, cudaStreamWaitEvent(st, iv.done, 0));
@@ -554,7 +567,8 @@ int ffn_status(cep_plan* p) {
   if (q != cudaSuccess) return fail(p, CEP_ERR_CUDA, "cudaEventQuery failed: %s", cudaGetErrorString(q));
   if (hs[kStTimeout]) return fail(p, CEP_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired");
   if (hs[kStBoundsViolation]) return fail(p, CEP_ERR_CAPACITY, "a row index left the scratch slot (more local pairs than planned)");
-  if (hs[kStBadRouting]) return fail(p, CEP_ERR_BAD_ROUTING, "an expert id was outside [0, n_experts_global)");
+  if (hs[kStBadRouting] & 1) return fail(p, CEP_ERR_BAD_ROUTING, "an expert id was outside [0, n_experts_global)");
+  if (hs[kStBadRouting] & 2) return fail(p, CEP_ERR_BAD_ROUTING, "a token names the same expert in two of its slots");
   return CEP_OK;
 }
 

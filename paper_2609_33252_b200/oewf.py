@@ -1,4 +1,4 @@
-"""Host-only simulation of opportunistic expert weight fetching (Section 4.2; Algorithm 1; Eqs. 1-6; the
+"""Host-only simulation of opportunistic expert weight fetching (Section 3.3 "Opportunistic Expert Weight Fetching"; Algorithm 1; Eqs. 1-6; the
 non-degradation proposition of the appendix).
 
 Nothing here touches a GPU or moves weights: cross-GPU fetching is outside what this library runs.  The module

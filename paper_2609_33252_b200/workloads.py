@@ -7,7 +7,7 @@ e4m3) and the chunk / arrival schedule.  It contains none of the arithmetic of t
 path itself (no permutation, no expert FFN, no combine) and is the one module the
 CUDA path's harnesses and the CPU oracle's tests both use.
 
-Inputs stand in for the serving traces the paper evaluates on (Section 5 setup):
+Inputs stand in for the serving traces the paper evaluates on ("Evaluation Settings", workloads):
 those traces are not available, so every tensor is synthetic and seeded.
 
 Representation: all tensors are torch tensors on ``device``.  bf16 tensors are
@@ -82,7 +82,7 @@ CONFIGS = {
                                  chunks=tuple(_equal_chunks(2048, 8)), dtype="fp8", zipf_s=1.1),
     "fp8_shard": MoEConfig("fp8_shard", 4, T=32768, H=7168, I=3072, E_global=512, E_local=64, k=8,
                            chunks=tuple(_equal_chunks(32768, 8)), dtype="fp8", zipf_s=1.1),
-    # microscaling variant of the EP shard (Section 5.1: MXFP4 routed-expert weights): same shapes and routing
+    # microscaling variant of the EP shard ("Evaluation Settings", models and environments: MXFP4 routed-expert weights): same shapes and routing
     "mxfp4_tiny": MoEConfig("mxfp4_tiny", 5, T=256, H=512, I=256, E_global=8, E_local=8, k=2,
                             chunks=(160, 96), dtype="mxfp4"),
     "mxfp4_shard_small": MoEConfig("mxfp4_shard_small", 5, T=2048, H=7168, I=2048, E_global=64, E_local=8, k=8,

@@ -243,6 +243,56 @@ def test_error_paths():
     assert e.value.code == -3
 
 
+def test_chunk_coverage_and_alignment_are_checked_on_the_host():
+    # return codes only: nothing that could write out of bounds is ever launched
+    cfg = wl.CONFIGS["tiny"]
+    host = wl.make_inputs(cfg)
+    inp = to_device(host)
+    layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC)
+    load(layer, inp)
+    out = torch.zeros(cfg.T + 8, cfg.H, dtype=torch.bfloat16, device="cuda")
+    ch = chunks_of(inp)
+    with pytest.raises(cep.CepError) as e:                 # output rows are stored 16 bytes at a time
+        cep.ffn_begin(layer.plan, out.view(-1)[1:], cfg.T, 2)
+    assert e.value.code == -1
+    cep.ffn_begin(layer.plan, out, cfg.T, 2)
+    cep.ffn_submit_chunk(layer.plan, 0, 0, 160, ch[0][1], None, ch[0][3], ch[0][4])
+    with pytest.raises(cep.CepError) as e:                 # overlaps chunk 0: 160 + 156 tokens > 256
+        cep.ffn_submit_chunk(layer.plan, 1, 100, 156, inp.x[100:256], None, inp.topk_ids[100:256], inp.topk_w[100:256])
+    assert e.value.code == -4
+    # a short last chunk leaves rows uncovered: reported, the submitted work still completes
+    cep.ffn_submit_chunk(layer.plan, 1, 160, 90, inp.x[160:250], None, inp.topk_ids[160:250], inp.topk_w[160:250])
+    assert cep.ffn_flush(layer.plan, allow_incomplete=True) == -5
+    assert cep.combine(layer.plan, allow_incomplete=True) == -5
+    torch.cuda.synchronize()
+    assert cep.ffn_status(layer.plan) == 0
+    check_close(out[:250], oracle.from_inputs(host, sel=np.arange(250)), "short coverage")
+    layer.close()
+
+
+def test_duplicate_expert_in_a_token_is_reported_by_debug_plans():
+    cfg = wl.CONFIGS["tiny"]
+    host = wl.make_inputs(cfg)
+    inp = to_device(host)
+    dup = inp.topk_ids.clone()
+    dup[7, 1] = dup[7, 0]
+    out = torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
+    for debug, want in ((1, -6), (0, 0)):
+        layer = make_layer(cfg, mode=cep.CEP_MODE_SYNC, debug_checks=debug)
+        load(layer, inp)
+        cep.ffn_begin(layer.plan, out, cfg.T, 1)
+        cep.ffn_submit_chunk(layer.plan, 0, 0, cfg.T, inp.x, None, dup, inp.topk_w)
+        cep.combine(layer.plan)
+        torch.cuda.synchronize()
+        assert cep.ffn_status(layer.plan) == want
+        if debug:
+            assert "same expert" in cep.cep_last_error(layer.plan)
+            assert cep.cep_debug_check_guards(layer.plan) == 0
+            out2, _ = run_layer(inp, layer)                  # clean ids: clean status, right answer
+            check_close(out2, oracle.from_inputs(host), "after duplicate ids")
+        layer.close()
+
+
 def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
     # failure detection without a fault: a wait that nothing satisfies runs out after its limit, the kernel
     # exits normally, the host reads CEP_ERR_DEVICE_TIMEOUT, and the next layer call is clean and correct

@@ -4,11 +4,14 @@ Who needs it: code that runs where device memory is already spoken for (a plug-i
 process whose pool owns the GPU) or where allocating is not allowed at that moment.  Such a caller
 passes only its own pre-made input and output buffers; the library's scratch is a fixed array inside
 the library.  The test makes two calls in a row on different inputs (the array keeps the first call's
-contents) and compares every integer with what the plan-based path exports for the same ids.
+contents) and compares every integer with what the plan-based path exports for the same ids, and
+with the CPU oracle's layout transform directly.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2609_33252_b200 as cep
 from paper_2609_33252_b200 import workloads as wl
 
@@ -56,6 +59,49 @@ def test_noalloc_layout_matches_plan_path_on_two_calls_in_a_row():
         assert (b["rop"].cpu().numpy() == ref["row_of_pair"]).all()
         n_rows = int(ref["padded_offsets"][-1])
         assert (b["por"][:n_rows].cpu().numpy() == ref["pair_of_row"]).all()   # padding rows stay -1
+        # and against the oracle itself, so this check does not lean on the plan path being right
+        want = oracle.permute(c.topk_ids.cpu().numpy(), c.cfg.E_local, align=128)
+        assert (b["counts"].cpu().numpy() == want["counts"]).all()
+        assert (b["offsets"].cpu().numpy() == want["offsets"]).all()
+        assert (b["padded"].cpu().numpy() == want["padded_offsets"]).all()
+        assert (b["rop"].cpu().numpy() == want["prow_of_pair"]).all()
+        assert (b["por"][:n_rows].cpu().numpy() == want["pair_of_prow"]).all()
+
+
+def test_noalloc_reports_bad_ids_and_a_short_inverse_map_without_touching_memory_past_it():
+    i32 = dict(dtype=torch.int32, device="cuda")
+    E, E_g, k, T = 4, 6, 2, 300
+    g = torch.Generator(device="cpu"); g.manual_seed(7)
+    ids = torch.stack([torch.randperm(E_g, generator=g)[:k] for _ in range(T)]).to(torch.int32)
+    want = oracle.permute(ids.numpy(), E, align=128)
+    n_rows = int(want["padded_offsets"][-1])
+
+    def call(ids_dev, por):
+        b = dict(counts=torch.zeros(E, **i32), offsets=torch.zeros(E + 1, **i32), padded=torch.zeros(E + 1, **i32),
+                 rop=torch.full((T * k,), -7, **i32), status=torch.full((2,), -7, **i32))
+        assert cep.layout_indices_noalloc(ids_dev, E, E_g, b["counts"], b["offsets"], b["padded"], b["rop"], por,
+                                          b["status"]) == 0
+        torch.cuda.synchronize()
+        return b
+    # (1) an id equal to n_experts_global: flagged in status[0], counted nowhere
+    bad = ids.clone(); bad[5, 1] = E_g
+    b = call(bad.cuda(), torch.full((n_rows,), -1, **i32))
+    assert b["status"].tolist() == [1, 0]
+    # (2) an inverse map shorter than the rows needed: status[1], rows that do not fit get -1 and are not stored;
+    #     the entries past the capacity handed in keep their sentinel
+    cap = n_rows - 200
+    assert cap > 0
+    store = torch.full((n_rows + 64,), 12345, **i32)
+    b = call(ids.cuda(), store[:cap])
+    assert b["status"].tolist() == [0, 1]
+    assert (store[cap:] == 12345).all()
+    rop, prow = b["rop"].cpu().numpy(), want["prow_of_pair"]
+    fits = (prow >= 0) & (prow < cap)
+    assert (rop[fits] == prow[fits]).all() and (rop[~fits] == -1).all()
+    got_por, want_por = store[:cap].cpu().numpy(), want["pair_of_prow"][:cap]
+    real = want_por >= 0
+    assert (got_por[real] == want_por[real]).all() and (got_por[~real] == 12345).all()   # padding rows are left untouched
+    assert (b["counts"].cpu().numpy() == want["counts"]).all()
 
 
 def test_noalloc_rejects_sizes_beyond_its_fixed_scratch_and_bad_arguments():
