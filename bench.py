@@ -26,12 +26,10 @@ if ROOT not in sys.path:
 METRIC = "MoE-layer prefill tokens/s (streamFFN routed-expert path: permute + grouped SwiGLU expert FFN + combine)"
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one GEMM1 launch, from the ncu captures summarised in
-# profiles/grouped_gemm_bf16_pair_ep_shard.md, profiles/grouped_gemm_fp8_pair_fp8_shard_small.md and
-# profiles/grouped_gemm_mx_pair_mxfp4_shard.md
-GEMM1_DRAM_TRAFFIC = {"ep_shard": 5.64e9 + 0.51e9, "straggler": 5.64e9 + 0.51e9,
-                      "ep_shard_small": 1.02e9 + 0.041e9, "fp8_shard_small": 0.462e9 + 0.034e9,
-                      "mxfp4_shard": 1.427e9 + 0.260e9, "mxfp4_shard_small": 0.204e9 + 0.019e9}
+# measured DRAM traffic of GEMM1 per launch: one record per workload, each naming the profiler command, date,
+# commit and the hash of the kernel source it was captured from
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "gemm1_dram_traffic.json")
+KERNEL_SOURCE = {"bf16": "gemm_tcgen05.cu", "fp8": "gemm_tcgen05_fp8.cu", "mxfp4": "gemm_tcgen05_mx.cu"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -48,18 +46,20 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons with nvidia-smi (a read-only query) while the timed region
+    runs.  The GPU is addressed by its UUID (an index would ignore CUDA_VISIBLE_DEVICES); every sample carries
+    the host time it was read at, and only samples taken between the region's two synchronisation points count."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, gpu_id: str):
+        self.gpu_id, self.rows, self.proc = gpu_id, [], None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -68,9 +68,9 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -78,18 +78,63 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
-            except Exception:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+        def fold(rows):
+            sm, mx, reasons, power = [], [], set(), []
+            for _, r in rows:
+                try:
+                    sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+                except Exception:
+                    continue
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            return sm, mx, reasons, power
+        # a sample is printed a little after it was taken: allow one sampling period of slack at the front
+        inside = [x for x in self.rows if t_begin + 0.02 <= x[0] <= t_end + 0.01]
+        sm, mx, reasons, power = fold(inside)
+        all_sm, all_mx, all_reasons, _ = fold(self.rows)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_mhz_min": min(sm) if sm else None,
+                "sm_max_mhz": max(all_mx) if all_mx else None,
+                "power_w_max": max(power) if power else None, "power_w_median": statistics.median(power) if power else None,
+                "samples": len(sm), "samples_outside_region": len(all_sm) - len(sm),
+                "reasons": sorted(reasons), "reasons_outside_region": sorted(all_reasons - reasons)}
+
+
+def gpu_identifier(local_rank: int) -> str:
+    import torch
+    try:
+        u = str(torch.cuda.get_device_properties(local_rank).uuid)
+        return u if u.startswith("GPU-") else "GPU-" + u
+    except Exception:
+        return str(local_rank)
+
+
+def sha256_of(path: str) -> str:
+    import hashlib
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def recorded_traffic(cfg):
+    """GEMM1's measured DRAM bytes per launch for this workload, if a capture of the CURRENT kernel source is on
+    record; (None, reason) otherwise."""
+    try:
+        with open(TRAFFIC_RECORD) as f:
+            rec = json.load(f)
+    except Exception:
+        return None, "no traffic record"
+    ent = rec.get(cfg.name)
+    if ent is None:
+        return None, "no capture of this workload on record"
+    src = KERNEL_SOURCE[cfg.dtype]
+    now = sha256_of(os.path.join(ROOT, "paper_2609_33252_b200", "csrc", src))
+    if ent.get("source_sha256", {}).get(src) != now:
+        return None, "%s changed since the capture of %s (commit %s)" % (src, ent.get("date"), ent.get("commit"))
+    return float(ent["dram_bytes_read"]) + float(ent["dram_bytes_write"]), \
+        "ncu capture of %s, commit %s%s" % (ent.get("date"), ent.get("commit"),
+                                           (", " + ent["note"]) if ent.get("note") else "")
 
 
 def workload_numbers(cfg, n_pairs):
@@ -171,18 +216,22 @@ def run_reference(args):
 
 def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
     """Completion latency of Sync / Async / Async+streamFFN when the chunks arrive at seeded offsets
-    (lognormal, scaled to tau x the one-shot time), and the matched-work retention at tau = 0."""
+    (lognormal, scaled to tau x the one-shot time), the matched-work retention at tau = 0, and the gate
+    "chunked asynchronous execution is no slower than one synchronous launch over the same tokens"."""
     import torch
     from paper_2609_33252_b200.arrivals import run_with_arrivals
     theta = args.theta if args.theta >= 0 else cfg.E_local * 1024
     rstreams = [torch.cuda.Stream() for _ in chunks]
-    modes = [("sync", cep.CEP_MODE_SYNC, 0, 1), ("async", cep.CEP_MODE_ASYNC, 0, 1),
-             ("streamffn", cep.CEP_MODE_STREAMFFN, theta, args.streams)]
+    # streamffn: the launch rule as the paper states it; streamffn_defer: a batch that has reached theta while the
+    # GPU is still busy with the previous invocation keeps accumulating (cep_config::defer_while_busy)
+    modes = [("sync", cep.CEP_MODE_SYNC, 0, 1, 0), ("async", cep.CEP_MODE_ASYNC, 0, 1, 0),
+             ("streamffn", cep.CEP_MODE_STREAMFFN, theta, args.streams, 0),
+             ("streamffn_defer", cep.CEP_MODE_STREAMFFN, theta, args.streams, 1)]
     layers = {}
-    for name, mode, th, S in modes:
+    for name, mode, th, S, defer in modes:
         L = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, mode=mode,
                          dtype=cep.DTYPE_OF[cfg.dtype],
-                         n_streams=S, threshold_pairs=th, gemm_impl=args.gemm_impl)
+                         n_streams=S, threshold_pairs=th, gemm_impl=args.gemm_impl, defer_while_busy=defer)
         L.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
         layers[name] = L
     torch.cuda.synchronize()
@@ -192,16 +241,33 @@ def stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, t_sync_s, args):
     for tau in (0.0, 0.25, 0.5, 1.0):
         arr = [tau * t_sync_s * a for a in base]
         case = {"tau": tau, "last_arrival_ms": max(arr) * 1e3}
-        for name, _, _, _ in modes:
-            ts, ninv = [], 0
-            for rep in range(13):                  # 3 warm-up + 10 timed
-                dt, ninv = run_with_arrivals(layers[name], out, chunks, arr, ch_pairs, rstreams)
+        # the modes take turns inside every repetition, so that all of them see the same clock and power state
+        ts = {name: [] for name, _, _, _, _ in modes}
+        ninv = {}
+        for rep in range(13):                      # 3 warm-up + 10 timed
+            for name, _, _, _, _ in modes:
+                dt, ninv[name] = run_with_arrivals(layers[name], out, chunks, arr, ch_pairs, rstreams)
                 if rep >= 3:
-                    ts.append(dt)
-            case[name] = {"completion_ms": statistics.median(ts) * 1e3, "min_ms": min(ts) * 1e3, "invocations": ninv}
+                    ts[name].append(dt)
+        for name, _, _, _, _ in modes:
+            case[name] = {"completion_ms": statistics.median(ts[name]) * 1e3, "min_ms": min(ts[name]) * 1e3,
+                          "invocations": ninv[name]}
         report["cases"].append(case)
     c0 = report["cases"][0]
-    report["matched_work_retention"] = {m: c0["sync"]["completion_ms"] / c0[m]["completion_ms"] for m in ("async", "streamffn")}
+    report["matched_work_retention"] = {m: c0["sync"]["completion_ms"] / c0[m]["completion_ms"]
+                                        for m in ("async", "streamffn", "streamffn_defer")}
+    staggered = report["cases"][1:]
+    report["gate"] = {
+        "statement": "completion latency of chunked asynchronous execution <= one synchronous launch over the same "
+                     "tokens, for every staggered arrival pattern (tau > 0); at tau = 0 (everything present at once) "
+                     "the synchronous launch is the best possible schedule and the retention is reported instead",
+        "streamffn_no_slower_than_sync": {str(c["tau"]): bool(c["streamffn"]["completion_ms"] <= c["sync"]["completion_ms"])
+                                          for c in staggered},
+        "streamffn_defer_no_slower_than_sync": {str(c["tau"]): bool(c["streamffn_defer"]["completion_ms"] <= c["sync"]["completion_ms"])
+                                                for c in staggered},
+        "retention_at_tau0": {"streamffn": report["matched_work_retention"]["streamffn"],
+                              "streamffn_defer": report["matched_work_retention"]["streamffn_defer"],
+                              "paper_other_system_and_hardware": 0.973}}
     for L in layers.values():
         L.close()
     return report
@@ -221,6 +287,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stream", action="store_true", help="skip the arrival-offset (streamFFN) section")
     ap.add_argument("--theta", type=int, default=-1, help="streamFFN threshold in local pairs (default: E_local*1024)")
+    ap.add_argument("--profile-in-region", type=int, default=-1,
+                    help="1: the timed plan itself records events between its kernels, so the per-kernel times come from "
+                         "the timed steps; 0: a second plan is profiled after the timed region; default: 1 for workloads "
+                         "of at least 2 TFLOP per step (the events cost a few microseconds of launch overlap per step)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3 if args.impl == "ours" else args.warmup
@@ -255,13 +325,17 @@ def main():
     ch_pairs = [int((inp.topk_ids[o:o + n] < cfg.E_local).sum().item()) for o, n in zip(inp.chunk_offsets, cfg.chunks)]
 
     dt = cep.DTYPE_OF[cfg.dtype]
+    in_region = args.profile_in_region == 1 or (args.profile_in_region < 0 and work["flops"] >= 2e12)
     layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
-                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, gemm_impl=args.gemm_impl)
+                         mode=cep.CEP_MODE_SYNC, n_streams=args.streams, gemm_impl=args.gemm_impl,
+                         profile_kernels=1 if in_region else 0)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
-    # a second plan that records events between the kernels: per-kernel device times, outside the timed region
-    prof_layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
-                              mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1, gemm_impl=args.gemm_impl)
-    prof_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
+    prof_layer = None
+    if not in_region:
+        # small workloads: a second plan records events between the kernels, run right after the timed region
+        prof_layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
+                                  mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1, gemm_impl=args.gemm_impl)
+        prof_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     torch.cuda.synchronize()
     out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
     chunks = [(o, inp.x[o:o + n], None if inp.x_scale is None else inp.x_scale[o:o + n], inp.topk_ids[o:o + n],
@@ -280,24 +354,31 @@ def main():
     barrier()
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
 
-    kern = {"layout_ms": [], "gemm1_ms": [], "gemm2_ms": [], "combine_ms": [], "index_ms": [], "scatter_ms": []}
+    names = ("layout_ms", "gemm1_ms", "gemm2_ms", "combine_ms", "index_ms", "scatter_ms", "elapsed_ms")
+    kern = {k_: [] for k_ in names}
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     bad_reasons = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+    gpu_id = gpu_identifier(local_rank)
     for attempt in range(2):            # a run that saw a thermal or hardware slowdown is taken once more
-        sampler = ClockSampler(local_rank)
+        sampler = ClockSampler(gpu_id)
         if rank == 0:
             sampler.start()
-            time.sleep(0.3)
+            time.sleep(0.1)
         launches0 = cep.cep_kernel_launches(layer.plan)
         barrier()
+        t_begin = time.time()
+        step_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
         ev0.record()
-        for _ in range(args.steps):
+        for i in range(args.steps):
             step()
+            step_ev[i].record()                    # the join stream: complete when this step's output is
         ev1.record()
         barrier()
+        t_end = time.time()
         total_ms = ev0.elapsed_time(ev1)
+        step_ms = [(ev0 if i == 0 else step_ev[i - 1]).elapsed_time(step_ev[i]) for i in range(args.steps)]
         launches = cep.cep_kernel_launches(layer.plan) - launches0
-        timed_clocks = sampler.stop() if rank == 0 else None
+        timed_clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
         redo = 1 if (rank == 0 and timed_clocks and bad_reasons & set(timed_clocks.get("reasons", []))) else 0
         if dist is not None:
             flag = torch.tensor([redo], device="cuda")
@@ -306,17 +387,25 @@ def main():
         if not redo:
             break
     assert cep.ffn_status(layer.plan) == 0, cep.cep_last_error(layer.plan)
-    # per-kernel times: a few more steps, each followed by a sync and a query (outside the timed region)
-    # per-kernel device times: the profiled plan runs the same number of steps back to back (same clocks and
-    # thermal state as the timed region); the plan keeps the events of its last layer call, read after a sync
-    for rep in range(3):
-        for _ in range(max(args.steps // 3, 1)):
-            prof_layer.run(out, chunks, n_local_pairs=ch_pairs)
-        torch.cuda.synchronize()
-        for i in range(cep.ffn_num_invocations(prof_layer.plan)):
-            info = cep.ffn_query(prof_layer.plan, i)
-            for k_ in kern:
-                kern[k_].append(getattr(info, k_))
+    if in_region:
+        # the plan keeps the events of its last layer calls: per-kernel device times of the last timed steps themselves
+        kernel_source = "events recorded between the kernels of the last %d timed steps" % min(args.steps, 8)
+        for back in range(min(args.steps, 8)):
+            for i in range(cep.ffn_num_invocations(layer.plan)):
+                info = cep.ffn_query_call(layer.plan, back, i)
+                for k_ in kern:
+                    kern[k_].append(getattr(info, k_))
+    else:
+        kernel_source = "a second, event-instrumented plan run back to back right after the timed region (the timed " \
+                        "plan records no events: they would cost this short step its launch overlap)"
+        for rep in range(3):
+            for _ in range(max(args.steps // 3, 1)):
+                prof_layer.run(out, chunks, n_local_pairs=ch_pairs)
+            torch.cuda.synchronize()
+            for i in range(cep.ffn_num_invocations(prof_layer.plan)):
+                info = cep.ffn_query(prof_layer.plan, i)
+                for k_ in kern:
+                    kern[k_].append(getattr(info, k_))
     clocks = timed_clocks
     if clocks is not None:
         clocks["remeasured"] = attempt == 1
@@ -430,7 +519,8 @@ def main():
     if rank == 0 and not args.no_stream and cfg.n_chunks > 1:
         stream_report = stream_section(cep, wl, cfg, inp, out, chunks, ch_pairs, ms * 1e-3, args)
 
-    prof_layer.close()
+    if prof_layer is not None:
+        prof_layer.close()
     if rank != 0:
         layer.close()
         if dist is not None:
@@ -443,26 +533,38 @@ def main():
     ffn_tflops = work["flops"] / ((g1_ms + g2_ms) * 1e-3) / 1e12
     g1_tflops = work["gemm1_flops"] / (g1_ms * 1e-3) / 1e12
     g2_tflops = work["gemm2_flops"] / (g2_ms * 1e-3) / 1e12
-    # burst peak for a short timed region at full clocks; sustained peak once the steps run under the power cap
-    # (cap reported active, clock well below maximum, or more than a second of back-to-back steps)
+    # Which measured peak the fraction is taken of: the burst figure for a short region at full clocks, the
+    # sustained one once the steps ran under the power cap (cap reported by a sample INSIDE the region, its median
+    # clock well below the maximum, or more than a second of back-to-back steps).  The power controller needs on
+    # the order of 100 ms of load before it pulls the clocks down.  All three fractions are printed side by side.
     sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
     capped = "sw_power_cap" in ((clocks or {}).get("reasons") or [])
-    # (the power controller needs on the order of 100 ms of load before it pulls the clocks down: a timed region
-    # shorter than that ran at burst clocks whatever the sampled flags say)
     sustained = total_ms > 100.0 and (capped or total_ms > 1000.0 or bool(sm and smx and sm < 0.9 * smx))
-    peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-    nominal_tf = NOMINAL_BF16_TFLOPS
-    if cfg.dtype in ("fp8", "mxfp4"):   # no measured fp8 peak: the measured bf16 peak times the nominal fp8/bf16 ratio (2);
-        #                                 the mxf8f6f4 MMA kind (e4m3 x e2m1) runs at the fp8 rate
-        peak_tf, nominal_tf = 2.0 * peak_tf, 2.0 * NOMINAL_BF16_TFLOPS
+    mult = 2.0 if cfg.dtype in ("fp8", "mxfp4") else 1.0   # no measured fp8 peak: measured bf16 peak x the nominal fp8:bf16
+    #                                                        ratio; the mxf8f6f4 MMA kind (e4m3 x e2m1) runs at the fp8 rate
+    burst_tf, sust_tf, nominal_tf = mult * peaks["bf16_tflops"], mult * peaks["bf16_tflops_sustained"], mult * NOMINAL_BF16_TFLOPS
+    peak_tf = sust_tf if sustained else burst_tf
+    traffic, traffic_note = recorded_traffic(cfg)
+    kernel_sum = sum(med[k_] for k_ in ("layout_ms", "gemm1_ms", "gemm2_ms", "combine_ms"))
     roofline = {"bound": "tensor", "kernel": "grouped GEMM1 (gate/up + SiLU*up%s), CTA-pair tcgen05" %
                           (" + e4m3 re-quantisation" if cfg.dtype != "bf16" else ""),
                 "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
                 "peak_kind": ("sustained" if sustained else "burst") + " bf16 cuBLAS" +
                              (" x2 (nominal fp8:bf16 ratio)" if cfg.dtype != "bf16" else "") + ", of " + peaks["source"],
+                "frac_of_burst": g1_tflops / burst_tf, "frac_of_sustained": g1_tflops / sust_tf,
                 "frac_of_nominal": g1_tflops / nominal_tf, "nominal_tflops": nominal_tf,
-                "duration_ms": g1_ms, "traffic": None}
-    roofline["traffic"] = GEMM1_DRAM_TRAFFIC.get(cfg.name)
+                "duration_ms": g1_ms, "share_of_step": g1_ms / ms, "traffic": traffic, "traffic_source": traffic_note,
+                "algorithmic_bytes": work["gemm1_bytes"]}
+    n_last = min(args.steps, 8)
+    last_ms = statistics.median(step_ms[-n_last:])          # the steps the per-kernel times were read from
+    timing = {"timed_region_ms": total_ms, "kernel_times_from": kernel_source,
+              "kernel_sum_ms": kernel_sum, "invocation_elapsed_ms": med["elapsed_ms"],
+              "ms_per_step_first": step_ms[0], "ms_per_step_median": statistics.median(step_ms),
+              "ms_per_step_median_of_last_%d" % n_last: last_ms,
+              "kernel_sum_within_those_steps": bool(kernel_sum <= last_ms * 1.005) if in_region else None,
+              "note": "the first steps of a region run at burst clocks, the later ones under the power cap: ms_per_step "
+                      "is the mean over all timed steps, the per-kernel times are medians over the last ones",
+              "sm_mhz_median_in_region": sm, "ms_per_step_x_sm_mhz": (ms * sm) if sm else None}
     kernels = {
         "layout": {"ms": med["layout_ms"], "GB/s": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9,
                    "frac_of_hbm": work["layout_bytes"] / (med["layout_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
@@ -484,7 +586,7 @@ def main():
                              (3.0 * cfg.H * cfg.I * {"bf16": 2, "fp8": 1, "mxfp4": 0.5}[cfg.dtype] * cfg.E_local / 1e9)},
             "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal": ffn_tflops / nominal_tf, "nominal_tflops": nominal_tf,
                            "frac_of_measured": ffn_tflops / peak_tf, "flops_per_step": work["flops"]},
-            "roofline": roofline, "kernels": kernels, "clocks": clocks, "e2e": e2e, "streamffn": stream_report,
+            "roofline": roofline, "timing": timing, "kernels": kernels, "clocks": clocks, "e2e": e2e, "streamffn": stream_report,
             "gpu_launches": int(launches)}
     if not args.no_cpu_baseline:
         import oracle

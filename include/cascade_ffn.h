@@ -120,7 +120,15 @@ typedef struct {
                                   status word instead of trapping                               */
   int32_t profile_kernels;     /* nonzero: record CUDA events between the kernels of every
                                   invocation so ffn_query can report per-kernel device times    */
-  int32_t reserved_;           /* set to 0                                                      */
+  int32_t defer_while_busy;    /* CEP_MODE_STREAMFFN only.  0: a batch is launched the moment it reaches
+                                  theta (the launch rule as Section 3.2 states it).  Nonzero: when theta
+                                  is reached while the previous invocation of this layer call is still
+                                  running on the GPU, the launch is put off and chunks keep accumulating:
+                                  queued work gains nothing from being split, and fewer, larger batches
+                                  keep the expert GEMMs efficient.  The batch goes out at the first later
+                                  ffn_submit_chunk that finds that invocation finished, when it holds
+                                  4*theta pairs or CEP_MAX_CHUNKS_PER_INVOCATION chunks, or at the flush.
+                                  Batching then depends on GPU timing (results do not)             */
 } cep_config;
 
 /* Per-invocation record for tracing (ffn_query). */
@@ -182,7 +190,7 @@ CEP_API int ffn_begin(cep_plan* plan, void* out, int32_t n_tokens_total, int32_t
 /*
  * Optional, between ffn_begin and the first ffn_submit_chunk: `addend` [device] bf16 [n_tokens_total, H] in
  * token order is added to every output row (fp32, before the single rounding).  This is the shared expert's
- * output: the combine result "is added to the shared-expert output" (Appendix "Output return and combine").
+ * output, which the layer sums with the routed result (Appendix "Output return and combine").
  * The rows of a chunk's tokens must be complete on that chunk's stream when the chunk is submitted.  NULL
  * (the default after ffn_begin) adds nothing.
  */
@@ -251,6 +259,14 @@ CEP_API int ffn_num_invocations(const cep_plan* plan);
 CEP_API int ffn_query(cep_plan* plan, int32_t inv, cep_invocation_info* info);
 
 /*
+ * The same record for an earlier layer call: calls_back = 0 is the current (or last) call, 1 the one before,
+ * up to 7 for plans made with profile_kernels (other plans keep only the current call: CEP_ERR_ARG).  Lets a
+ * harness run several layer calls back to back without a host synchronisation in between and read every call's
+ * per-kernel device times afterwards.  pairs_bound and the chunk fields are those of that call.
+ */
+CEP_API int ffn_query_call(cep_plan* plan, int32_t calls_back, int32_t inv, cep_invocation_info* info);
+
+/*
  * Copy the layout transform's integers of invocation `inv` to [host] arrays (any may be
  * NULL): counts[E], offsets[E+1], padded_offsets[E+1], row_of_pair[n_tokens*k] (physical,
  * tile-aligned row of each pair in batch pair order, -1 if not local), pair_of_row[
@@ -305,6 +321,19 @@ typedef struct {
 CEP_API int cep_calibrate(cep_plan* plan, float rho, const int32_t* rows_per_expert, int32_t n_points, int32_t reps,
                           const void* tokens, const void* token_scales, int32_t* ids, float* weights, void* out,
                           cep_profile_point* points, cep_calibration* result);
+
+/*
+ * The same calibration on the CALLER'S routing: the profile is taken on growing prefixes of one real batch
+ * (the first n_tokens[i] tokens of tokens / ids / weights, ascending, each run as one synchronous invocation),
+ * so theta reflects the expert skew the layer actually sees: with a skewed router the unpopular experts of a
+ * batch get far fewer rows than the mean, and an invocation reaches a given throughput only at a larger
+ * expert-token count than uniform routing suggests.  points[i].expert_tokens is the number of local
+ * (token, expert) pairs in that prefix, rows_per_expert their mean per local expert.  No stream probe
+ * (best_streams = 0).  Same requirements as cep_calibrate; ids and weights are read, not written.
+ */
+CEP_API int cep_calibrate_routed(cep_plan* plan, float rho, const int32_t* n_tokens, int32_t n_points, int32_t reps,
+                                 const void* tokens, const void* token_scales, const int32_t* ids, const float* weights,
+                                 void* out, cep_profile_point* points, cep_calibration* result);
 
 /* Total kernel launches this plan has issued (layout, GEMM, combine, prepack). */
 CEP_API int64_t cep_kernel_launches(const cep_plan* plan);

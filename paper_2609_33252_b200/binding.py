@@ -25,7 +25,7 @@ EXPORTS = ["moe_plan_workspace_bytes", "moe_packed_weight_bytes", "moe_plan", "m
            "ffn_begin", "ffn_submit_chunk", "ffn_flush", "combine", "ffn_status", "ffn_num_invocations",
            "ffn_query", "ffn_debug_export", "cep_kernel_launches", "moe_plan_destroy", "cep_last_error",
            "cep_debug_decode_tile", "cep_debug_schedule", "layout_indices_noalloc", "cep_debug_wait_timeout", "ffn_set_addend", "moe_route", "cep_debug_check_guards", "ffn_wait_invocation",
-           "ffn_set_active_streams", "cep_calibrate"]
+           "ffn_set_active_streams", "cep_calibrate", "ffn_query_call", "cep_calibrate_routed"]
 
 
 class CepConfig(ctypes.Structure):
@@ -35,7 +35,7 @@ class CepConfig(ctypes.Structure):
                 ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("n_streams", ctypes.c_int32),
                 ("threshold_pairs", ctypes.c_int64), ("gemm_impl", ctypes.c_int32),
                 ("debug_checks", ctypes.c_int32), ("profile_kernels", ctypes.c_int32),
-                ("reserved_", ctypes.c_int32)]
+                ("defer_while_busy", ctypes.c_int32)]
 
 
 class InvocationInfo(ctypes.Structure):
@@ -97,6 +97,7 @@ def load_library(build_if_missing: bool = True):
         "ffn_num_invocations": (ctypes.c_int, [vp]),
         "ffn_wait_invocation": (ctypes.c_int, [vp, i32, vp]),
         "ffn_query": (ctypes.c_int, [vp, i32, ctypes.POINTER(InvocationInfo)]),
+        "ffn_query_call": (ctypes.c_int, [vp, i32, i32, ctypes.POINTER(InvocationInfo)]),
         "ffn_debug_export": (ctypes.c_int, [vp, i32, vp, vp, vp, vp, vp]),
         "cep_kernel_launches": (i64, [vp]),
         "moe_plan_destroy": (ctypes.c_int, [vp]),
@@ -110,6 +111,8 @@ def load_library(build_if_missing: bool = True):
         "ffn_set_active_streams": (ctypes.c_int, [vp, i32]),
         "cep_calibrate": (ctypes.c_int, [vp, ctypes.c_float, vp, i32, i32, vp, vp, vp, vp, vp,
                                          ctypes.POINTER(ProfilePoint), ctypes.POINTER(Calibration)]),
+        "cep_calibrate_routed": (ctypes.c_int, [vp, ctypes.c_float, vp, i32, i32, vp, vp, vp, vp, vp,
+                                                ctypes.POINTER(ProfilePoint), ctypes.POINTER(Calibration)]),
         "layout_indices_noalloc": (ctypes.c_int, [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -215,6 +218,12 @@ def ffn_query(plan, inv: int) -> InvocationInfo:
     return info
 
 
+def ffn_query_call(plan, calls_back: int, inv: int) -> InvocationInfo:
+    info = InvocationInfo()
+    _check(lib().ffn_query_call(plan, calls_back, inv, ctypes.byref(info)), plan)
+    return info
+
+
 def ffn_debug_export(plan, inv: int, n_experts_local: int, n_pairs: int):
     """Returns dict of numpy int32 arrays: counts, offsets, padded_offsets, row_of_pair, pair_of_row."""
     import numpy as np
@@ -246,6 +255,19 @@ def cep_calibrate(plan, rho: float, rows_per_expert: Sequence[int], reps: int, t
     points = [{f: getattr(p, f) for f, _ in ProfilePoint._fields_} for p in pts]
     result = {f: getattr(cal, f) for f, _ in Calibration._fields_ if f != "stream_ms"}
     result["stream_ms"] = [v for v in cal.stream_ms if v >= 0]
+    return points, result
+
+
+def cep_calibrate_routed(plan, rho: float, n_tokens: Sequence[int], reps: int, tokens, token_scales, ids, weights, out):
+    """Calibration on the caller's routing: profile on growing prefixes of one real batch (see the header)."""
+    n = len(n_tokens)
+    nt = (ctypes.c_int32 * n)(*[int(v) for v in n_tokens])
+    pts = (ProfilePoint * n)()
+    cal = Calibration()
+    _check(lib().cep_calibrate_routed(plan, float(rho), ctypes.cast(nt, ctypes.c_void_p), n, reps, _dptr(tokens),
+                                      _dptr(token_scales), _dptr(ids), _dptr(weights), _dptr(out), pts, ctypes.byref(cal)), plan)
+    points = [{f: getattr(p, f) for f, _ in ProfilePoint._fields_} for p in pts]
+    result = {f: getattr(cal, f) for f, _ in Calibration._fields_ if f != "stream_ms"}
     return points, result
 
 
@@ -316,12 +338,13 @@ class MoELayer:
 
     def __init__(self, hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
                  dtype=CEP_BF16, mode=CEP_MODE_STREAMFFN, n_streams=2, threshold_pairs=0,
-                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, profile_kernels=0, device="cuda"):
+                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, profile_kernels=0, defer_while_busy=0, device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the streamFFN library needs a CUDA device; there is no CPU path")
         self.cfg = CepConfig(hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
-                             dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks, profile_kernels, 0)
+                             dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks, profile_kernels,
+                             defer_while_busy)
         self.device = torch.device(device)
         self.workspace = torch.empty(moe_plan_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
         self.packed = torch.empty(moe_packed_weight_bytes(self.cfg), dtype=torch.uint8, device=self.device)

@@ -2,7 +2,7 @@
 // contribution is weighted by its routing coefficient exactly once and accumulated at its
 // token; results are written in token order.  Slots are accumulated in ascending slot
 // order in fp32 and rounded to bf16 once.  Tokens with no local expert get exact zeros.  An optional addend
-// row (the shared expert's output for the token: "the result is added to the shared-expert output") is added
+// row (the shared expert's output for the token, which the paper sums with the routed result) is added
 // in fp32 after the routed contributions, before the single rounding.
 #include <cuda_bf16.h>
 

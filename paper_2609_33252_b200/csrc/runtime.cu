@@ -19,6 +19,7 @@ namespace {
 thread_local char g_error[256] = "";          // last error of a call that had no plan to record it in
 constexpr int kGuardByte = 0xA5;
 constexpr size_t kStatusBlockBytes = 256;        // one status block (kStWords int32) per layer-call parity
+constexpr int kTraceCalls = 8;                   // profile_kernels: layer calls whose per-kernel events are kept
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -150,9 +151,15 @@ struct cep_plan {
   std::vector<cudaStream_t> streams;
   std::vector<Slot> slots;
   std::vector<cudaEvent_t> ready_evt;           // per chunk position
-  std::vector<Invocation> inv;
-  std::vector<cudaEvent_t> inv_start, inv_done; // pools, one per possible invocation
+  std::vector<Invocation> inv;                  // the current (or last) layer call
+  // Event pools: one set per possible invocation of a layer call.  With profile_kernels there are kTraceCalls
+  // sets, used in turn, and `past` keeps the records of the calls before the current one, so per-kernel device
+  // times of several back-to-back layer calls can be read after they have all run (ffn_query_call).
+  std::vector<cudaEvent_t> inv_start, inv_done;
   std::vector<cudaEvent_t> inv_mark;            // 4 per possible invocation (profile_kernels)
+  std::vector<Invocation> past[kTraceCalls];
+  int trace_sets;                               // 1, or kTraceCalls with profile_kernels
+  long long call_index;                         // layer calls opened so far
   // Two status blocks, used by alternate layer calls: a call clears its block without waiting for the previous
   // call's read-back (a small device-to-host copy that can sit behind the caller's own output copies in the copy
   // engine's queue), only for the read-back of the call before that.
@@ -188,7 +195,8 @@ int launch_invocation(cep_plan* p) {
   if (p->pending.empty()) return CEP_OK;
   const cep_config& c = p->cfg;
   const int idx = (int)p->inv.size();
-  if (idx >= (int)p->inv_start.size()) return fail(p, CEP_ERR_CAPACITY, "more invocations than max_chunks");
+  if (idx >= c.max_chunks) return fail(p, CEP_ERR_CAPACITY, "more invocations than max_chunks");
+  const int ev = (int)(p->call_index % p->trace_sets) * c.max_chunks + idx;      // this call's set of events
   const int slot_i = idx % p->active_streams;
   Slot& sl = p->slots[slot_i];
   cudaStream_t st = p->streams[slot_i];
@@ -208,10 +216,10 @@ int launch_invocation(cep_plan* p) {
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->begin_evt, 0));
   CUDA_TRY(p, cudaStreamWaitEvent(st, p->weights_evt, 0));
   for (size_t i = 0; i < p->pending.size(); ++i) CUDA_TRY(p, cudaStreamWaitEvent(st, p->ready_evt[first_pos + (int)i], 0));
-  Invocation iv{first_pos, batch.n_chunks, slot_i, tok, p->pending_pairs, p->inv_start[idx], p->inv_done[idx],
+  Invocation iv{first_pos, batch.n_chunks, slot_i, tok, p->pending_pairs, p->inv_start[ev], p->inv_done[ev],
                 {nullptr, nullptr, nullptr, nullptr}, false};
   const bool prof = c.profile_kernels != 0 && tok > 0;
-  if (prof) { for (int m = 0; m < 4; ++m) iv.mark[m] = p->inv_mark[4 * idx + m]; iv.profiled = true; }
+  if (prof) { for (int m = 0; m < 4; ++m) iv.mark[m] = p->inv_mark[4 * ev + m]; iv.profiled = true; }
   CUDA_TRY(p, cudaEventRecord(iv.start, st));
   if (tok > 0) {
     const long long n_pairs = (long long)tok * c.top_k;
@@ -326,6 +334,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   p->err[0] = 0; p->launches = 0; p->active_streams = cfg->n_streams;
   p->have_weights = p->layer_open = p->flushed = p->ever_closed = false;
   p->readback_pending[0] = p->readback_pending[1] = false; p->status_idx = 0;
+  p->trace_sets = cfg->profile_kernels ? kTraceCalls : 1; p->call_index = -1;
   p->host_status = nullptr; p->begin_evt = p->readback_evt[0] = p->readback_evt[1] = p->weights_evt = nullptr;
   p->out = nullptr; p->addend = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
   int dev = 0;
@@ -347,6 +356,9 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   for (int i = 0; i < cfg->max_chunks; ++i) {
     cudaEvent_t e;
     PLAN_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming)); p->ready_evt.push_back(e);
+  }
+  for (int i = 0; i < cfg->max_chunks * p->trace_sets; ++i) {
+    cudaEvent_t e;
     PLAN_TRY(cudaEventCreate(&e)); p->inv_start.push_back(e);
     PLAN_TRY(cudaEventCreate(&e)); p->inv_done.push_back(e);
     if (cfg->profile_kernels)
@@ -462,6 +474,8 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   p->out = out; p->addend = nullptr; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
   p->n_submitted = 0; p->tokens_submitted = 0;
   p->chunk_seen.assign(n_chunks_expected, 0);
+  if (p->call_index >= 0) p->past[p->call_index % kTraceCalls] = p->inv;    // the call that just ended
+  p->call_index += 1;
   p->pending.clear(); p->pending_pairs = 0; p->inv.clear();
   p->layer_open = true; p->flushed = false;
   return CEP_OK;
@@ -500,8 +514,16 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   p->chunk_seen[chunk_id] = 1;
   p->n_submitted += 1;
   p->tokens_submitted += n_tokens;
-  if (should_launch(p->cfg.mode, p->pending_pairs, (int)p->pending.size(), p->cfg.threshold_pairs))
+  if (should_launch(p->cfg.mode, p->pending_pairs, (int)p->pending.size(), p->cfg.threshold_pairs)) {
+    // Work that would only queue behind a running invocation is not split off: see cep_config::defer_while_busy.
+    if (p->cfg.defer_while_busy && p->cfg.mode == CEP_MODE_STREAMFFN && !p->inv.empty() &&
+        (int)p->pending.size() < kMaxChunksPerInv && p->pending_pairs < 4 * p->cfg.threshold_pairs) {
+      const cudaError_t q = cudaEventQuery(p->inv.back().done);
+      if (q == cudaErrorNotReady) { (void)cudaGetLastError(); return CEP_OK; }
+      if (q != cudaSuccess) return fail(p, CEP_ERR_CUDA, "cudaEventQuery failed: %s", cudaGetErrorString(q));
+    }
     return launch_invocation(p);
+  }
   return CEP_OK;
 }
 
@@ -581,10 +603,7 @@ int ffn_wait_invocation(cep_plan* p, int32_t inv, void* stream) {
 
 int ffn_num_invocations(const cep_plan* p) { return p ? (int)p->inv.size() : CEP_ERR_ARG; }
 
-int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {
-  if (!p || !info) return fail(p, CEP_ERR_ARG, "NULL argument");
-  if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
-  const Invocation& iv = p->inv[inv];
+static void fill_info(const Invocation& iv, cep_invocation_info* info) {
   info->n_chunks = iv.n_chunks; info->first_chunk_pos = iv.first_pos; info->stream_index = iv.slot;
   info->n_tokens = iv.n_tokens; info->pairs_bound = iv.pairs_bound; info->elapsed_ms = -1.f;
   info->layout_ms = info->gemm1_ms = info->gemm2_ms = info->combine_ms = info->index_ms = info->scatter_ms = -1.f;
@@ -600,6 +619,23 @@ int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {
       if (cudaEventElapsedTime(&ms, iv.mark[2], iv.done) == cudaSuccess) info->combine_ms = ms;
     }
   }
+}
+
+int ffn_query(cep_plan* p, int32_t inv, cep_invocation_info* info) {
+  if (!p || !info) return fail(p, CEP_ERR_ARG, "NULL argument");
+  if (inv < 0 || inv >= (int)p->inv.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist", inv);
+  fill_info(p->inv[inv], info);
+  return CEP_OK;
+}
+
+int ffn_query_call(cep_plan* p, int32_t calls_back, int32_t inv, cep_invocation_info* info) {
+  if (!p || !info) return fail(p, CEP_ERR_ARG, "NULL argument");
+  if (calls_back == 0) return ffn_query(p, inv, info);
+  if (calls_back < 0 || calls_back >= p->trace_sets || calls_back > p->call_index)
+    return fail(p, CEP_ERR_ARG, "the records of %d layer calls ago are not kept", calls_back);
+  const std::vector<Invocation>& v = p->past[(p->call_index - calls_back) % kTraceCalls];
+  if (inv < 0 || inv >= (int)v.size()) return fail(p, CEP_ERR_ARG, "invocation %d does not exist in that layer call", inv);
+  fill_info(v[inv], info);
   return CEP_OK;
 }
 
@@ -747,6 +783,64 @@ int cep_calibrate(cep_plan* p, float rho, const int32_t* rows_per_expert, int32_
 #undef CAL_TRY
 #undef CAL_CUDA
   restore();
+  return CEP_OK;
+}
+
+int cep_calibrate_routed(cep_plan* p, float rho, const int32_t* n_tokens, int32_t n_points, int32_t reps,
+                         const void* tokens, const void* token_scales, const int32_t* ids, const float* weights,
+                         void* out, cep_profile_point* points, cep_calibration* res) {
+  if (!p) return fail(nullptr, CEP_ERR_ARG, "plan is NULL");
+  if (!n_tokens || !tokens || !ids || !weights || !out || !points || !res) return fail(p, CEP_ERR_ARG, "a calibration pointer is NULL");
+  if (!(rho > 0.f && rho <= 1.f) || n_points < 1 || reps < 1 || reps > 100) return fail(p, CEP_ERR_ARG, "need 0 < rho <= 1, n_points >= 1, 1 <= reps <= 100");
+  if (p->layer_open) return fail(p, CEP_ERR_STATE, "cep_calibrate_routed while a layer call is open");
+  if (!p->have_weights) return fail(p, CEP_ERR_STATE, "cep_calibrate_routed before moe_load_weights");
+  if (!p->cfg.profile_kernels) return fail(p, CEP_ERR_STATE, "cep_calibrate_routed needs a plan made with profile_kernels != 0");
+  for (int i = 0; i < n_points; ++i)
+    if (n_tokens[i] < 1 || (i > 0 && n_tokens[i] <= n_tokens[i - 1]) || n_tokens[i] > p->cfg.max_tokens)
+      return fail(p, CEP_ERR_ARG, "n_tokens must be positive, ascending and at most max_tokens");
+  const int saved_mode = p->cfg.mode;
+  const int E = p->cfg.n_experts_local;
+  cudaStream_t s0 = p->streams[0];
+  p->cfg.mode = CEP_MODE_SYNC;
+  int rc = CEP_OK;
+  float peak = 0.f;
+  for (int i = 0; i < n_points && rc == CEP_OK; ++i) {
+    const int T = n_tokens[i];
+    std::vector<float> ffn, layer;
+    int32_t n_local = 0;
+    for (int r = 0; r < reps + 2 && rc == CEP_OK; ++r) {
+      rc = ffn_begin(p, out, T, 1);
+      if (rc == CEP_OK) rc = ffn_submit_chunk(p, 0, 0, T, tokens, token_scales, ids, weights, -1, s0);
+      if (rc == CEP_OK) rc = combine(p, s0);
+      if (rc == CEP_OK && cudaStreamSynchronize(s0) != cudaSuccess) rc = fail(p, CEP_ERR_CUDA, "cudaStreamSynchronize failed");
+      if (rc == CEP_OK) rc = ffn_status(p);
+      cep_invocation_info info;
+      if (rc == CEP_OK) rc = ffn_query(p, 0, &info);
+      if (rc == CEP_OK && r >= 2) { ffn.push_back(info.gemm1_ms + info.gemm2_ms); layer.push_back(info.elapsed_ms); }
+    }
+    // the expert tokens of this prefix of the batch: the last entry of the offsets the layout transform just made
+    if (rc == CEP_OK && cudaMemcpy(&n_local, p->slots[p->inv[0].slot].lp.offsets + E, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+      rc = fail(p, CEP_ERR_CUDA, "cudaMemcpy of the pair count failed");
+    if (rc != CEP_OK) break;
+    cep_profile_point& pt = points[i];
+    pt.n_tokens = T; pt.expert_tokens = n_local; pt.rows_per_expert = n_local / E;
+    pt.ffn_ms = median_of(ffn); pt.layer_ms = median_of(layer);
+    pt.tflops = pt.ffn_ms > 0.f ? (float)(6.0 * p->cfg.hidden * p->cfg.inter * (double)n_local / (pt.ffn_ms * 1e-3) / 1e12) : 0.f;
+    pt.eta = 0.f;
+    if (pt.tflops > peak) peak = pt.tflops;
+  }
+  p->cfg.mode = saved_mode;
+  if (rc != CEP_OK) {
+    if (p->layer_open) { p->pending.clear(); p->pending_pairs = 0; p->layer_open = false; }
+    return rc;
+  }
+  res->rho = rho; res->peak_tflops = peak;
+  res->theta_pairs = points[n_points - 1].expert_tokens; res->theta_rows_per_expert = points[n_points - 1].rows_per_expert;
+  for (int i = 0; i < n_points; ++i) points[i].eta = peak > 0.f ? points[i].tflops / peak : 0.f;
+  for (int i = 0; i < n_points; ++i)
+    if (points[i].eta >= rho) { res->theta_pairs = points[i].expert_tokens; res->theta_rows_per_expert = points[i].rows_per_expert; break; }
+  for (int s = 0; s < 16; ++s) res->stream_ms[s] = -1.f;
+  res->best_streams = 0; res->probe_invocations = 0;
   return CEP_OK;
 }
 

@@ -3,7 +3,7 @@ non-degradation proposition of the appendix).
 
 Nothing here touches a GPU or moves weights: cross-GPU fetching is outside what this library runs.  The module
 restates the planner's decisions so that they can be exercised with this library's own FFN latency profile
-(``calibrate.calibrate`` gives eta(N) and the observed peak) and synthetic attention / dispatch times:
+(``calibrate.calibrate_in_library`` / ``calibrate_on_routing`` give eta(N) and the observed peak) and synthetic attention / dispatch times:
 
 * ``FFNLatency``            F(N) = N / (eta(N) * P_peak), F(0) = 0                       (Eq. 2)
 * ``remaining_attention``   A_d = [f(I_d, P_d) - t_att]^+                                 (Eq. 1)
@@ -75,21 +75,20 @@ def select_weights(helper: int, donors_T: Dict[int, float], tokens_h: Dict[int, 
     attention); tokens_h[d][e]: tokens helper h dispatched to expert e of donor d; budget: B_h.  The donor
     with the latest completion is chosen; its experts that hold tokens of h are taken in descending
     tokens-per-byte order while they fit, stopping at the first that does not."""
-    if not donors_T:
+    import itertools
+    ranked_donors = sorted(donors_T.items(), key=lambda kv: (-kv[1], kv[0]))      # latest completion first, ties: lowest rank
+    if not ranked_donors:
         return None
-    donor = max(sorted(donors_T), key=lambda d: donors_T[d])           # ties: lowest rank id
-    eligible = [e for e, n in tokens_h.get(donor, {}).items() if n > 0]
-    order = sorted(eligible, key=lambda e: (-tokens_h[donor][e] / bytes_per_expert[e], e))
-    chosen, remaining = [], budget
-    for e in order:
-        if bytes_per_expert[e] <= remaining:
-            chosen.append(e)
-            remaining -= bytes_per_expert[e]
-        else:
-            break
-    if not chosen:
+    donor = ranked_donors[0][0]
+    held = tokens_h.get(donor, {})
+    density_order = sorted((e for e in held if held[e] > 0), key=lambda e: (-held[e] / bytes_per_expert[e], e))
+    # running byte total over the density-ordered experts; the selection is the longest prefix within the budget
+    running = list(itertools.accumulate(bytes_per_expert[e] for e in density_order))
+    n_fit = sum(1 for _ in itertools.takewhile(lambda total: total <= budget, running))
+    if n_fit == 0:
         return None
-    return FetchPlan(helper, donor, chosen, {e: tokens_h[donor][e] for e in chosen}, budget - remaining)
+    chosen = density_order[:n_fit]
+    return FetchPlan(helper, donor, chosen, {e: held[e] for e in chosen}, running[n_fit - 1])
 
 
 def overlap_fraction(T_h: float, s_h: float, F_trans: float) -> float:

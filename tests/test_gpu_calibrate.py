@@ -81,3 +81,64 @@ def test_active_streams_changes_the_slots_not_the_result():
         with pytest.raises(cep.CepError):
             cep.ffn_set_active_streams(layer.plan, bad)
     layer.close()
+
+
+def test_calibration_on_the_callers_routing_counts_the_real_expert_tokens():
+    # growing prefixes of one skewed batch: expert_tokens are the local pairs of each prefix, theta the first
+    # profiled count that reaches rho of the best throughput seen on THIS routing
+    cfg = wl.scaled(CFG, zipf_s=1.1)
+    res = calibrate.calibrate_on_routing(cfg, rho=0.9, fractions=(1 / 16, 1 / 4, 1.0), reps=3)
+    host_ids = wl.make_inputs(cfg, device="cuda", keep_logits=False).topk_ids.cpu().numpy()
+    prof = res["profile"]
+    assert [p["n_tokens"] for p in prof] == [128, 512, 2048]
+    for p in prof:
+        assert p["expert_tokens"] == int((host_ids[:p["n_tokens"]] < cfg.E_local).sum())
+        assert p["ffn_ms"] > 0 and 0 < p["eta"] <= 1.0 + 1e-6
+    reach = [p for p in prof if p["eta"] >= 0.9]
+    assert res["theta_pairs"] == reach[0]["expert_tokens"] and res["best_streams"] == 0
+
+
+def test_per_kernel_times_of_earlier_layer_calls_are_kept():
+    cfg = wl.scaled(CFG, chunks=(1024, 1024))
+    inp = to_device(wl.make_inputs(cfg))
+    layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, 2, mode=cep.CEP_MODE_ASYNC, n_streams=2,
+                         profile_kernels=1)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+    out = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16, device="cuda")
+    from helpers import chunks_of
+    for _ in range(5):                                            # back to back, no host synchronisation in between
+        layer.run(out, chunks_of(inp))
+    torch.cuda.synchronize()
+    for back in range(5):
+        for i in range(2):
+            q = cep.ffn_query_call(layer.plan, back, i)
+            assert q.n_tokens == 1024 and q.first_chunk_pos == i
+            assert q.elapsed_ms > 0 and q.gemm1_ms > 0 and q.gemm2_ms > 0 and q.combine_ms > 0
+            assert q.layout_ms + q.gemm1_ms + q.gemm2_ms + q.combine_ms == pytest.approx(q.elapsed_ms, rel=1e-3, abs=1e-3)
+    with pytest.raises(cep.CepError):
+        cep.ffn_query_call(layer.plan, 5, 0)                      # only five calls were made
+    with pytest.raises(cep.CepError):
+        cep.ffn_query_call(layer.plan, 8, 0)                      # never kept
+    layer.close()
+    plain = make_layer(cfg)                                       # plans without profile_kernels keep the current call only
+    plain.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+    run_layer(inp, plain); run_layer(inp, plain)
+    with pytest.raises(cep.CepError):
+        cep.ffn_query_call(plain.plan, 1, 0)
+    plain.close()
+
+
+def test_deferring_launches_while_the_gpu_is_busy_changes_batching_not_results():
+    cfg = wl.scaled(CFG, chunks=(256,) * 8)
+    inp = to_device(wl.make_inputs(cfg))
+    pairs = int((inp.topk_ids[:256] < cfg.E_local).sum().item())
+    outs, n_inv = [], []
+    for defer in (0, 1):
+        layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, 8, mode=cep.CEP_MODE_STREAMFFN, n_streams=2,
+                             threshold_pairs=pairs, defer_while_busy=defer)
+        layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+        o, n = run_layer(inp, layer, local_pairs=True)
+        outs.append(o); n_inv.append(n)
+        layer.close()
+    assert 1 <= n_inv[1] <= n_inv[0]                              # never more invocations than the plain threshold rule
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))

@@ -1,6 +1,6 @@
 """The steps either side of the routed-expert path: the router kernel in front (softmax, top-k, renormalise;
 ids bit-exact against the oracle's routing, ties to the lower id) and the shared expert's output added by the
-combine (Appendix "Output return and combine": the result is added to the shared-expert output)."""
+combine (Appendix "Output return and combine": routed result and shared-expert output are summed)."""
 import numpy as np
 import pytest
 import torch
