@@ -91,6 +91,10 @@ CONFIGS = {
                                  chunks=(1404,) * 7 + (16384 - 7 * 1404,), dtype="mxfp4", zipf_s=1.1, straggler_last=True),
     "mxfp4_shard": MoEConfig("mxfp4_shard", 5, T=16384, H=7168, I=2048, E_global=256, E_local=32, k=8,
                              chunks=tuple(_equal_chunks(16384, 8)), dtype="mxfp4", zipf_s=1.1),
+    # one EP rank's shard of the larger MXFP4 model of the paper's model table ("Evaluation Settings": 384 routed
+    # experts per layer, 6 per token, expert intermediate size 3072); the hidden size is not in the paper: 7168 assumed
+    "mxfp4_pro_shard": MoEConfig("mxfp4_pro_shard", 6, T=16384, H=7168, I=3072, E_global=384, E_local=48, k=6,
+                                 chunks=tuple(_equal_chunks(16384, 8)), dtype="mxfp4", zipf_s=1.1),
 }
 
 

@@ -40,7 +40,7 @@ def sample_tokens(inp, n_random=40, seed=0):
     return np.unique(np.array(sel, dtype=np.int64))
 
 
-@pytest.mark.parametrize("name", ["ep_shard", "ep_shard_strided", "mxfp4_shard", "fp8_shard"])
+@pytest.mark.parametrize("name", ["ep_shard", "ep_shard_strided", "mxfp4_shard", "fp8_shard", "mxfp4_pro_shard"])
 def test_ep_shard_full_size(name):
     cfg = wl.CONFIGS[name]
     inp = wl.make_inputs(cfg, device="cuda", keep_logits=False)
