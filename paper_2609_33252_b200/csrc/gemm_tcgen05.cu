@@ -495,6 +495,20 @@ int make_operand_map(GemmTensorMap* out, const void* base, int elt_bytes, int K,
   return r == CUDA_SUCCESS ? 0 : -2;
 }
 
+int make_store_map(GemmTensorMap* out, void* base, int elt_bytes, int cols, long long rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return -1;
+  CUtensorMap* m = reinterpret_cast<CUtensorMap*>(out);
+  const CUtensorMapDataType dt = elt_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * elt_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(64 / elt_bytes), 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -2;
+}
+
 int gemm_tile_rows() { return BM; }
 int gemm_tile_cols() { return BN; }
 

@@ -32,8 +32,11 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& 
 // tiles; pair == 0: one CTA per 128x256 tile.  The weight map's box has gemm_fp8_box_rows(pair) rows (the weight
 // rows one CTA loads per stage).
 int gemm_fp8_box_rows(int pair);
+// Output of the block-scaled kernels as the TMA engine stores it: a rows x cols tensor of elt_bytes elements
+// written in boxes of 32 rows x 64 bytes (64-byte swizzle in shared memory).
+int make_store_map(GemmTensorMap* out, void* base, int elt_bytes, int cols, long long rows);
 cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                            const float* a_scales, const float* b_scales, void* out, float* out_scales,
+                            const GemmTensorMap& tm_out, const float* a_scales, const float* b_scales, void* out, float* out_scales,
                             const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches);
 // s13p[e][2*ib + (0 gate | 1 up)][kb] and s2p[e][hb][kb] from the caller's [E, in/128, out/128] scale tensors
 cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const float* s_up, const float* s_down,

@@ -52,7 +52,7 @@ template <bool kPair> struct Geo {
   static constexpr int kRingReaders = kPair ? 20 : 11;    // producer, 2 MMA issuers, 8 promotion warps (+ peer: producer, 8)
   static constexpr int kPartArrivals = kPair ? 16 : 8;
   static constexpr int kSmemBytes = kStages * (A_STAGE + B_STAGE) + kBarBytes + (1024 + 1) * 4 + 12 + 2 * 2 * BM * 4 +
-                                    kPromoWarps * kStoreStage + 1024;
+                                    kPromoWarps * kStoreStage + 512 + 1024;
 };
 constexpr int kMaxStages = 6;
 constexpr int kThreads = 384;
@@ -158,29 +158,34 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
   return r;
 }
 
-// A warp holds 64 bytes of output per lane (lane = row).  Written to global memory directly, every store
-// instruction would touch 32 rows with 16 bytes each; staged through 2 KiB of shared memory (16-byte chunks
-// swizzled by row so that neither side has bank conflicts) each instruction covers 64 contiguous bytes of 8 rows.
-// Rows at or beyond n_rows are not stored.  dst = address of row 0, row_stride in bytes.
-__device__ __forceinline__ void store_rows_64B(uint8_t* stage, int lane, const uint4 (&ch)[4], uint8_t* dst,
-                                               size_t row_stride, int n_rows) {
+// A warp holds 64 bytes of output per lane (lane = row).  Written to global memory by the threads, every store
+// instruction would touch 32 rows with 16 bytes each and the tile's 64 KiB would queue in the load/store unit while
+// the MMAs wait for these warps.  Instead the warp lays its 32 x 64 bytes out in 2 KiB of shared memory (16-byte
+// chunk index XOR row bits: the TMA engine's 64-byte swizzle, which also keeps the writes free of bank conflicts)
+// and one lane hands the box to the TMA engine, which writes it out on its own.  The box covers all 32 rows: the
+// caller skips warps whose rows lie wholly beyond the expert's count (they may belong to the next expert); rows
+// between the count and the end of the expert's 128-row block are padding and receive the zeros computed for them.
+__device__ __forceinline__ void stage_rows_64B(uint8_t* stage, int lane, const uint4 (&ch)[4]) {
 #pragma unroll
   for (int q = 0; q < 4; ++q)
     *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) = ch[q];
-  __syncwarp();
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = 8 * i + (lane >> 2), c = lane & 3;
-    const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 64 + ((c ^ ((r >> 1) & 3)) << 4));
-    if (r < n_rows) *reinterpret_cast<uint4*>(dst + (size_t)r * row_stride + c * 16) = v;
-  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the writes, as the TMA engine must see them
   __syncwarp();
 }
+__device__ __forceinline__ void tma_store_box(const CUtensorMap* map, const uint8_t* stage, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(stage)) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the staging buffer may be overwritten again (the engine has read it)
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// every store of this thread has reached global memory
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 template <bool kSwiglu, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                             int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
+                             const __grid_constant__ CUtensorMap tm_out, int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
                              const float* __restrict__ a_scales /*[rows, num_kb]*/,
                              const float* __restrict__ b_scales /*[E, N/128, num_kb]*/,
                              uint8_t* __restrict__ out_codes, float* __restrict__ out_scales /*[rows, out cols/128]*/,
@@ -198,7 +203,8 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
   Bars* bars = reinterpret_cast<Bars*>(smem + kStages * (A_STAGE + B_STAGE));
   int32_t* pair_prefix = reinterpret_cast<int32_t*>(smem + kStages * (A_STAGE + B_STAGE) + kBarBytes);
   float* s_amax = reinterpret_cast<float*>(pair_prefix + kMaxExperts + 4);           // [tile parity][half][128]
-  uint8_t* s_store = reinterpret_cast<uint8_t*>(s_amax + 2 * 2 * BM);                // [promotion warp][kStoreStage]
+  // [promotion warp][kStoreStage], on a 512-byte boundary: the swizzle pattern is a function of the address bits
+  uint8_t* s_store = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(s_amax + 2 * 2 * BM) + 511) & ~(uintptr_t)511);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = kPair ? cluster_ctarank() : 0u;
   const bool is_peer = rank != 0;
@@ -459,12 +465,15 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
           }
           ch[q] = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        store_rows_64B(my_store, lane, ch, out_codes + (size_t)(tc.poff + r_warp) * out_ld + tc.n_block * 128 + 64 * half,
-                       (size_t)out_ld, tc.count - r_warp);
+        if (lane == 0) tma_store_wait_read();            // the previous tile's box has left the staging buffer
+        __syncwarp();
+        if (r_warp < tc.count) {
+          stage_rows_64B(my_store, lane, ch);
+          if (lane == 0) tma_store_box(&tm_out, my_store, tc.n_block * 128 + 64 * half, tc.poff + r_warp);
+        }
         if (half == 0 && row_ok) out_scales[grow * (n_out_cols / 128) + tc.n_block] = scale;
       } else {
         // 128 bf16 per row, 32 columns (64 bytes) per pass through the staging buffer
-        uint8_t* orow = reinterpret_cast<uint8_t*>(out_bf16 + (size_t)(tc.poff + r_warp) * out_ld + tc.n_block * BN + 128 * half);
 #pragma unroll
         for (int pass = 0; pass < 4; ++pass) {
           uint4 ch[4];
@@ -476,10 +485,16 @@ grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_c
             ch[q].z = pack_bf16(acc[i + 4], acc[i + 5]);
             ch[q].w = pack_bf16(acc[i + 6], acc[i + 7]);
           }
-          store_rows_64B(my_store, lane, ch, orow + 64 * pass, (size_t)out_ld * 2, tc.count - r_warp);
+          if (lane == 0) tma_store_wait_read();          // the previous box has left the staging buffer
+          __syncwarp();
+          if (r_warp < tc.count) {
+            stage_rows_64B(my_store, lane, ch);
+            if (lane == 0) tma_store_box(&tm_out, my_store, tc.n_block * BN + 128 * half + 32 * pass, tc.poff + r_warp);
+          }
         }
       }
     }
+    if (lane == 0) tma_store_wait_all();                 // this warp's boxes have reached global memory
   }
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
@@ -556,10 +571,10 @@ cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const
 }
 
 template <bool kSwiglu, bool kPair>
-static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, const CUtensorMap& b, int num_kb, int n_blocks_n,
+static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o, int num_kb, int n_blocks_n,
                               int n_group, int n_experts, int n_out_cols, int out_ld, const float* a_scales,
                               const float* b_scales, void* out, float* out_scales, const LayoutPtrs& lp, int32_t* counter) {
-  return cudaLaunchKernelEx(cfg, grouped_gemm_fp8_kernel<kSwiglu, kPair>, a, b, num_kb, n_blocks_n, n_group, n_experts,
+  return cudaLaunchKernelEx(cfg, grouped_gemm_fp8_kernel<kSwiglu, kPair>, a, b, o, num_kb, n_blocks_n, n_group, n_experts,
                             n_out_cols, out_ld, a_scales, b_scales, kSwiglu ? (uint8_t*)out : (uint8_t*)nullptr,
                             kSwiglu ? out_scales : (float*)nullptr, kSwiglu ? (__nv_bfloat16*)nullptr : (__nv_bfloat16*)out,
                             (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
@@ -569,7 +584,7 @@ static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, con
 // pair != 0: CTA pairs on 256x256 tiles, max_tiles counts pair tiles; pair == 0: one CTA per 128x256 tile,
 // max_tiles counts single tiles.  The weight operand map must have a box of gemm_fp8_box_rows(pair) rows.
 cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                            const float* a_scales, const float* b_scales, void* out, float* out_scales,
+                            const GemmTensorMap& tm_out, const float* a_scales, const float* b_scales, void* out, float* out_scales,
                             const LayoutPtrs& lp, int max_tiles, int n_sms, cudaStream_t s, int64_t* launches) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -607,7 +622,8 @@ cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap&
   cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
-#define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, p.out_ld, \
+  const CUtensorMap& o = reinterpret_cast<const CUtensorMap&>(tm_out);
+#define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, o, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, p.out_ld, \
                                                   a_scales, b_scales, out, out_scales, lp, counter)
   if (p.swiglu) e = pair ? CEP_FP8_LAUNCH(true, true) : CEP_FP8_LAUNCH(true, false);
   else e = pair ? CEP_FP8_LAUNCH(false, true) : CEP_FP8_LAUNCH(false, false);

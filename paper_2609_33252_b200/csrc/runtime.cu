@@ -29,6 +29,7 @@ struct Slot {
   uint8_t* act; void* act_scales;
   uint8_t* y;
   GemmTensorMap tm_a1, tm_a2;
+  GemmTensorMap tm_o1, tm_o2;                   // fp8: the intermediate and the down-projection output as store targets
   GemmTensorMap tm_sfa1, tm_sfa2;               // microscaling: scale atoms of the two activation operands
 };
 
@@ -250,11 +251,11 @@ int launch_invocation(cep_plan* p) {
       const int bn = gemm_tile_cols();
       const long long m_bound = pair ? (m_tiles_bound + groups + 1) / 2 : m_tiles_bound;
       const long long t1 = m_bound * ((g1.N + bn - 1) / bn), t2 = m_bound * ((g2.N + bn - 1) / bn);
-      CUDA_TRY(p, launch_gemm_fp8(g1, pair, sl.tm_a1, p->tm_b1, (const float*)sl.xp_scales, (const float*)p->s13p, sl.act,
+      CUDA_TRY(p, launch_gemm_fp8(g1, pair, sl.tm_a1, p->tm_b1, sl.tm_o1, (const float*)sl.xp_scales, (const float*)p->s13p, sl.act,
                                   (float*)sl.act_scales, sl.lp,
                                   (int)(t1 > (1 << 30) ? (1 << 30) : t1), p->n_sms, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
-      CUDA_TRY(p, launch_gemm_fp8(g2, pair, sl.tm_a2, p->tm_b2, (const float*)sl.act_scales, (const float*)p->s2p, sl.y, nullptr, sl.lp,
+      CUDA_TRY(p, launch_gemm_fp8(g2, pair, sl.tm_a2, p->tm_b2, sl.tm_o2, (const float*)sl.act_scales, (const float*)p->s2p, sl.y, nullptr, sl.lp,
                                   (int)(t2 > (1 << 30) ? (1 << 30) : t2), p->n_sms, st, &p->launches));
     } else if (c.gemm_impl == CEP_GEMM_TCGEN05) {
       const int bn = gemm_tile_cols();
@@ -384,6 +385,10 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     if (cfg->gemm_impl != CEP_GEMM_SIMT) {
       int r1 = make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
       int r2 = make_operand_map(&sl.tm_a2, sl.act, elt, cfg->inter, L.cap_rows, 0, gemm_tile_rows());
+      if (cfg->dtype == CEP_FP8_E4M3_BLOCK128 && !r1 && !r2) {
+        r1 = make_store_map(&sl.tm_o1, sl.act, 1, cfg->inter, L.cap_rows);
+        r2 = make_store_map(&sl.tm_o2, sl.y, 2, cfg->hidden, L.cap_rows);
+      }
       if (mx && !r1 && !r2) {
         r1 = make_mx_sf_map(&sl.tm_sfa1, sl.xp_scales, (long long)(L.cap_rows / kRowAlign) * (cfg->hidden / 128), kSfAtomBytes);
         r2 = make_mx_sf_map(&sl.tm_sfa2, sl.act_scales, (long long)(L.cap_rows / kRowAlign) * (cfg->inter / 128), kSfAtomBytes);
