@@ -9,9 +9,11 @@
 // warps pull every partial product out of tensor memory and add it, scaled, into fp32 accumulators
 // they hold in registers (128 per thread).
 //
-// What paces such a loop is the thread that issues the MMAs: every tcgen05 instruction (mma, commit) and
+// Two things pace such a loop.  The thread that issues the MMAs: every tcgen05 instruction (mma, commit) and
 // every barrier wait costs that one thread 60-100 cycles, and a K block here needs two waits (operands
-// landed, scratch buffer free) on top of its four MMAs, against 512 cycles of tensor work.  So the issue
+// landed, scratch buffer free) on top of its four MMAs, against 512 cycles of tensor work.  And the round
+// trip of a scratch buffer (MMAs complete -> promotion warps see it -> 128 values per thread read out ->
+// buffer handed back -> next MMA), of which only two can be in flight.  So the issue
 // is split over TWO threads, one per scratch buffer: K blocks alternate between them, each thread waits,
 // issues and commits for its own buffer only, and since every K block goes to its own buffer and the
 // promotion warps consume the buffers in K order, the result does not depend on how the two threads'
@@ -185,11 +187,11 @@ __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bu
 template <bool kSwiglu, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                             const __grid_constant__ CUtensorMap tm_out, int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
+                             const __grid_constant__ CUtensorMap tm_out /*codes (GEMM1) or bf16 (GEMM2), as boxes*/,
+                             int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols,
                              const float* __restrict__ a_scales /*[rows, num_kb]*/,
                              const float* __restrict__ b_scales /*[E, N/128, num_kb]*/,
-                             uint8_t* __restrict__ out_codes, float* __restrict__ out_scales /*[rows, out cols/128]*/,
-                             __nv_bfloat16* __restrict__ out_bf16,
+                             float* __restrict__ out_scales /*GEMM1: [rows, out cols/128]*/,
                              const int32_t* __restrict__ tile_prefix, const int32_t* __restrict__ counts,
                              const int32_t* __restrict__ padded_offsets, int32_t* __restrict__ tile_counter,
                              int32_t* __restrict__ status) {
@@ -572,11 +574,10 @@ cudaError_t launch_pack_scales(const cep_config& cfg, const float* s_gate, const
 
 template <bool kSwiglu, bool kPair>
 static cudaError_t launch_one(cudaLaunchConfig_t* cfg, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o, int num_kb, int n_blocks_n,
-                              int n_group, int n_experts, int n_out_cols, int out_ld, const float* a_scales,
-                              const float* b_scales, void* out, float* out_scales, const LayoutPtrs& lp, int32_t* counter) {
+                              int n_group, int n_experts, int n_out_cols, const float* a_scales,
+                              const float* b_scales, float* out_scales, const LayoutPtrs& lp, int32_t* counter) {
   return cudaLaunchKernelEx(cfg, grouped_gemm_fp8_kernel<kSwiglu, kPair>, a, b, o, num_kb, n_blocks_n, n_group, n_experts,
-                            n_out_cols, out_ld, a_scales, b_scales, kSwiglu ? (uint8_t*)out : (uint8_t*)nullptr,
-                            kSwiglu ? out_scales : (float*)nullptr, kSwiglu ? (__nv_bfloat16*)nullptr : (__nv_bfloat16*)out,
+                            n_out_cols, a_scales, b_scales, kSwiglu ? out_scales : (float*)nullptr,
                             (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets,
                             counter, lp.status);
 }
@@ -623,8 +624,9 @@ cudaError_t launch_gemm_fp8(const GemmProblem& p, int pair, const GemmTensorMap&
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
   const CUtensorMap& o = reinterpret_cast<const CUtensorMap&>(tm_out);
-#define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, o, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, p.out_ld, \
-                                                  a_scales, b_scales, out, out_scales, lp, counter)
+#define CEP_FP8_LAUNCH(SW, PR) launch_one<SW, PR>(&cfg, a, b, o, num_kb, n_blocks_n, n_group, p.n_experts, n_out_cols, \
+                                                  a_scales, b_scales, out_scales, lp, counter)
+  (void)out;                                             // the output tensor is reached through tm_out
   if (p.swiglu) e = pair ? CEP_FP8_LAUNCH(true, true) : CEP_FP8_LAUNCH(true, false);
   else e = pair ? CEP_FP8_LAUNCH(false, true) : CEP_FP8_LAUNCH(false, false);
 #undef CEP_FP8_LAUNCH
