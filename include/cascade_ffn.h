@@ -159,6 +159,11 @@ CEP_API int moe_packed_weight_bytes(const cep_config* cfg, size_t* bytes);
  * it is carved into S scratch slots (each invocation has its own scratch, Appendix
  * "Grouped FFN invocations") and stays owned by the caller.  Creates S non-blocking
  * streams and the events.  Must be called with the target device current.
+ * If the environment variable CEP_NVTX is set to anything but "" or "0" when the plan is made,
+ * the plan names its streams ("cep slot i") and wraps every layer call (ffn_begin .. combine) and
+ * every FFN invocation's enqueue in NVTX ranges, for timeline tools (the paper reads its attention
+ * and dispatch timings from such timelines, Appendix "Long-Tail Statistics of DEP Prefill"); without
+ * a tool attached the annotations do nothing.
  */
 CEP_API int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep_plan** out);
 

@@ -4,10 +4,14 @@
 // the device except in ffn_debug_export / ffn_query / moe_plan_destroy.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <algorithm>
 #include <new>
 #include <vector>
+
+#include <nvtx3/nvToolsExt.h>
+#include <nvtx3/nvToolsExtCudaRt.h>
 
 #include "cep_common.h"
 #include "gemm_tcgen05.h"
@@ -179,6 +183,8 @@ struct cep_plan {
   int64_t pending_pairs;
   int32_t* host_status;                         // pinned, two blocks of kStWords
   int64_t launches;
+  bool nvtx;                                    // CEP_NVTX=1 when the plan was made: ranges for timeline tools
+  nvtxRangeId_t call_range;
   char err[256];
 };
 
@@ -192,10 +198,24 @@ int fail(cep_plan* p, int code, const char* fmt, ...) {
 #define CUDA_TRY(p, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) \
   return fail((p), CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); } while (0)
 
+// A named range on the calling thread for as long as the object lives (only with CEP_NVTX=1).
+struct HostRange {
+  bool on;
+  HostRange(const cep_plan* p, const char* fmt, long long a, long long b, long long c) : on(p->nvtx) {
+    if (!on) return;
+    char name[96];
+    snprintf(name, sizeof name, fmt, a, b, c);
+    nvtxRangePushA(name);
+  }
+  ~HostRange() { if (on) nvtxRangePop(); }
+};
+
 int launch_invocation(cep_plan* p) {
   if (p->pending.empty()) return CEP_OK;
   const cep_config& c = p->cfg;
   const int idx = (int)p->inv.size();
+  HostRange range(p, "cep invocation %lld: %lld chunks, %lld expert tokens", idx, (long long)p->pending.size(),
+                  (long long)p->pending_pairs);
   if (idx >= c.max_chunks) return fail(p, CEP_ERR_CAPACITY, "more invocations than max_chunks");
   const int ev = (int)(p->call_index % p->trace_sets) * c.max_chunks + idx;      // this call's set of events
   const int slot_i = idx % p->active_streams;
@@ -338,6 +358,8 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
   p->trace_sets = cfg->profile_kernels ? kTraceCalls : 1; p->call_index = -1;
   p->host_status = nullptr; p->begin_evt = p->readback_evt[0] = p->readback_evt[1] = p->weights_evt = nullptr;
   p->out = nullptr; p->addend = nullptr; p->pending_pairs = 0; p->n_submitted = 0;
+  const char* nvtx_env = getenv("CEP_NVTX");
+  p->nvtx = nvtx_env && nvtx_env[0] && nvtx_env[0] != '0'; p->call_range = 0;
   int dev = 0;
 #define PLAN_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
     fail(nullptr, CEP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); moe_plan_destroy(p); return CEP_ERR_CUDA; } } while (0)
@@ -353,6 +375,7 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     cudaStream_t st;
     PLAN_TRY(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
     p->streams.push_back(st);
+    if (p->nvtx) { char name[32]; snprintf(name, sizeof name, "cep slot %d", s); nvtxNameCudaStreamA(st, name); }
   }
   for (int i = 0; i < cfg->max_chunks; ++i) {
     cudaEvent_t e;
@@ -483,6 +506,11 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   p->call_index += 1;
   p->pending.clear(); p->pending_pairs = 0; p->inv.clear();
   p->layer_open = true; p->flushed = false;
+  if (p->nvtx) {
+    char name[64];
+    snprintf(name, sizeof name, "cep layer call %lld: %d tokens", p->call_index, n_tokens_total);
+    p->call_range = nvtxRangeStartA(name);
+  }
   return CEP_OK;
 }
 
@@ -582,6 +610,7 @@ int combine(cep_plan* p, void* stream) {
   CUDA_TRY(p, cudaEventRecord(p->readback_evt[sb], st));
   p->readback_pending[sb] = true; p->ever_closed = true;
   p->layer_open = false;
+  if (p->nvtx) nvtxRangeEnd(p->call_range);
   return rc;
 }
 

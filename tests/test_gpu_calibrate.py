@@ -142,3 +142,20 @@ def test_deferring_launches_while_the_gpu_is_busy_changes_batching_not_results()
         layer.close()
     assert 1 <= n_inv[1] <= n_inv[0]                              # never more invocations than the plain threshold rule
     assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+
+
+def test_timeline_ranges_are_host_annotations_only(monkeypatch):
+    """CEP_NVTX=1 names the plan's streams and wraps layer calls and invocations in ranges for timeline tools; with no
+    tool attached the calls are no-ops and the output is bit-identical."""
+    cfg = wl.scaled(CFG, chunks=(256,) * 8)
+    inp = to_device(wl.make_inputs(cfg))
+    outs = []
+    for flag in ("0", "1"):
+        monkeypatch.setenv("CEP_NVTX", flag)
+        layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, 8, mode=cep.CEP_MODE_ASYNC, n_streams=2)
+        layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+        o, n = run_layer(inp, layer)
+        assert n == 8
+        outs.append(o)
+        layer.close()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
