@@ -129,6 +129,15 @@ typedef struct {
                                   ffn_submit_chunk that finds that invocation finished, when it holds
                                   4*theta pairs or CEP_MAX_CHUNKS_PER_INVOCATION chunks, or at the flush.
                                   Batching then depends on GPU timing (results do not)             */
+  int32_t gather_a;            /* bf16 with CEP_GEMM_TCGEN05 only (CEP_ERR_UNSUPPORTED otherwise).  Nonzero:
+                                  the layout transform (Appendix "Grouped FFN invocations") computes the
+                                  indices but moves no rows; the gate/up GEMM fetches each operand row
+                                  from the caller's tokens through a TMA row gather.  All chunks of a
+                                  layer call must then be row slices of ONE dense [n_tokens_total, H]
+                                  tensor (chunk pointer = tensor + token_offset rows; CEP_ERR_UNSUPPORTED
+                                  from ffn_submit_chunk otherwise), and that tensor must stay unchanged
+                                  until the layer call's combine work has run.  Results are bit-identical
+                                  to gather_a = 0; the workspace is smaller by the permuted copy      */
 } cep_config;
 
 /* Per-invocation record for tracing (ffn_query). */

@@ -35,7 +35,7 @@ class CepConfig(ctypes.Structure):
                 ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("n_streams", ctypes.c_int32),
                 ("threshold_pairs", ctypes.c_int64), ("gemm_impl", ctypes.c_int32),
                 ("debug_checks", ctypes.c_int32), ("profile_kernels", ctypes.c_int32),
-                ("defer_while_busy", ctypes.c_int32)]
+                ("defer_while_busy", ctypes.c_int32), ("gather_a", ctypes.c_int32)]
 
 
 class InvocationInfo(ctypes.Structure):
@@ -338,13 +338,14 @@ class MoELayer:
 
     def __init__(self, hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
                  dtype=CEP_BF16, mode=CEP_MODE_STREAMFFN, n_streams=2, threshold_pairs=0,
-                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, profile_kernels=0, defer_while_busy=0, device="cuda"):
+                 gemm_impl=CEP_GEMM_TCGEN05, debug_checks=0, profile_kernels=0, defer_while_busy=0, gather_a=0,
+                 device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the streamFFN library needs a CUDA device; there is no CPU path")
         self.cfg = CepConfig(hidden, inter, n_experts_global, n_experts_local, top_k, max_tokens, max_chunks,
                              dtype, mode, n_streams, threshold_pairs, gemm_impl, debug_checks, profile_kernels,
-                             defer_while_busy)
+                             defer_while_busy, gather_a)
         self.device = torch.device(device)
         self.workspace = torch.empty(moe_plan_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
         self.packed = torch.empty(moe_packed_weight_bytes(self.cfg), dtype=torch.uint8, device=self.device)

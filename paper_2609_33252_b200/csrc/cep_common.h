@@ -53,6 +53,7 @@ struct LayoutPtrs {
   int32_t* pair_of_row;       // [cap_rows] batch pair index, -1 on padding
   int32_t* status;            // [kStWords]
   int32_t* sched;             // [2] tile counters of the two GEMMs of an invocation (zeroed by the scan kernel)
+  int32_t* src_row;           // [cap_rows] gather_a plans only: row of the caller's token tensor a physical row holds
 };
 
 // ---------------------------------------------------------------- programmatic dependent launch

@@ -236,6 +236,12 @@ constexpr int kTilePoison = -2;
 constexpr int kSchedRing = 4;                          // tile ids in flight between the scheduler and its readers
 constexpr int kSchedReaders = 11;                      // leader: producer, MMA, 4 epilogue warps; peer: producer, 4 epilogue warps
 constexpr int kPairThreads = 224;                      // warp 6 of the leader CTA hands out tiles
+#ifndef CEP_GATHER_WARPS
+#define CEP_GATHER_WARPS 8
+#endif
+constexpr int kGatherWarps = CEP_GATHER_WARPS;         // gathering variant: warps 7.. of both CTAs fetch the activation rows
+constexpr int kGatherLanes = 32 / kGatherWarps;        // lanes of each that issue one four-row gather per stage
+constexpr int kPairThreadsGather = kPairThreads + 32 * kGatherWarps;
 struct __align__(8) PairBarriers {
   uint64_t full[kPairStages], empty[kPairStages], acc_full[2], acc_empty[2];
   uint64_t sched_full[kSchedRing], sched_empty[kSchedRing];
@@ -272,13 +278,17 @@ struct TileReader {
 constexpr int kPairSmemBytes = kPairStages * (A_STAGE + PB_STAGE) + (kMaxExperts + 1) * 4 + 1024 + 256;
 static_assert(sizeof(PairBarriers) <= 256, "barrier block");
 
-template <bool kSwiglu>
-__global__ void __launch_bounds__(kPairThreads, 1)
+// kGather: the activation operand is not the permuted copy but the caller's token tensor itself; tm_a then
+// describes that tensor with one-row boxes, src_row[r] is the tensor row that physical row r holds, and the
+// producer warp fetches every 128-row operand stage as 32 four-row gathers (one per lane).
+template <bool kSwiglu, bool kGather>
+__global__ void __launch_bounds__(kGather ? kPairThreadsGather : kPairThreads, 1)
 grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                               int num_kb, int n_blocks_n, int n_group, int n_experts, int n_out_cols, int out_ld,
                               __nv_bfloat16* __restrict__ out, const int32_t* __restrict__ tile_prefix,
                               const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
-                              int32_t* __restrict__ tile_counter, int32_t* __restrict__ status) {
+                              const int32_t* __restrict__ src_row, int32_t* __restrict__ tile_counter,
+                              int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   pdl_enter();
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -294,7 +304,7 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
     for (int s = 0; s < kPairStages; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), 8); }
     for (int s = 0; s < kSchedRing; ++s) {
-      mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders);
+      mbar_init(smem_u32(&bars->sched_full[s]), 1); mbar_init(smem_u32(&bars->sched_empty[s]), kSchedReaders + (kGather ? 2 * kGatherWarps : 0));
       bars->sched_tile[s] = kTilePoison;     // shared memory keeps what the previous CTA on this SM left
     }
     bars->abort_flag = 0;
@@ -342,7 +352,8 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
           // the leader alone arrives, announcing both CTAs' bytes; the peer's bytes can only land in
           // this phase because its loads wait for the stage to be freed by the leader's MMAs
           if (rank == 0) mbar_expect_tx(smem_u32(&bars->full[stage]), 2 * (A_STAGE + PB_STAGE));
-          tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * (BKB / 2), row0, full);
+          // (the gathering variant's activation rows are fetched by warps 7.., which wait for the stage themselves)
+          if constexpr (!kGather) tma_load_2d_pair(smem_u32(smem_a + stage * A_STAGE), &tm_a, kb * (BKB / 2), row0, full);
           tma_load_3d_pair(smem_u32(smem_b + stage * PB_STAGE), &tm_b, kb * (BKB / 2), n0, tc.expert, full);
           if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
         }
@@ -377,6 +388,49 @@ grouped_gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __
         if (!ok) break;
         tc_commit_pair_both(smem_u32(&bars->acc_full[acc]), 3);  // accumulator complete, both halves
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 7) {
+    // ---------------------------------------------------------------- row gather (kGather only; both CTAs)
+    // Warp g fetches rows [g, g+1) * 128/kGatherWarps of this CTA's operand block: its first kGatherLanes lanes
+    // issue one four-row gather each per stage.  The warp walks tiles and stages in lock-step behind lane 0,
+    // which does the waiting; the stage's byte count is announced by the producer warp of the leader CTA.
+    if constexpr (kGather) {
+      const int g = warp - 7;
+      int stage = 0; uint32_t phase = 0;
+      TileReader rd;
+      for (;;) {
+        int tile = -1;
+        if (lane == 0) { tile = rd.next(bars, is_peer, abort_flag, status); rd.done(bars, true); }
+        tile = __shfl_sync(0xffffffffu, tile, 0);
+        if (tile < 0) break;
+        TileCoord tc;
+        if (!decode_tile(pair_prefix, n_experts, n_blocks_n, n_group, tile, &tc)) break;
+        const int poff = padded_offsets[tc.expert], count = counts[tc.expert];
+        const int row_in_block = (g * kGatherLanes + lane) * 4;                       // first of this lane's four rows
+        const int r_local = tc.m_block * (2 * BM) + (int)rank * BM + row_in_block;
+        // Rows past the expert's count are padding: their products are never stored, so they re-read the
+        // expert's first row (always a real row) instead of an index that nothing wrote.
+        const int first = __ldg(src_row + poff);
+        int4 idx = make_int4(first, first, first, first);
+        if (lane < kGatherLanes && r_local < count) {
+          const int4 got = __ldg(reinterpret_cast<const int4*>(src_row + poff + r_local));
+          idx.x = got.x;
+          if (r_local + 1 < count) idx.y = got.y;
+          if (r_local + 2 < count) idx.z = got.z;
+          if (r_local + 3 < count) idx.w = got.w;
+        }
+        int ok = 1;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (lane == 0) ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status) ? 1 : 0;
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          if (lane < kGatherLanes)
+            tma_gather4_pair(smem_u32(smem_a + stage * A_STAGE + row_in_block * BKB), &tm_a, kb * (BKB / 2), idx,
+                             mapa(smem_u32(&bars->full[stage]), 0));
+          if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
       }
     }
   } else if (warp == 6) {
@@ -525,9 +579,11 @@ static cudaError_t current_device(int* dev) {
 
 static cudaError_t setup_pair_kernels(int dev, int n_sms) {
   if (g_pair_clusters[dev] > 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(grouped_gemm_bf16_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
@@ -536,16 +592,16 @@ static cudaError_t setup_pair_kernels(int dev, int n_sms) {
   cfg.gridDim = dim3(n_sms & ~1, 1, 1); cfg.blockDim = dim3(kPairThreads, 1, 1);
   cfg.dynamicSmemBytes = kPairSmemBytes; cfg.attrs = attr; cfg.numAttrs = 1;
   int n = 0;
-  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_bf16_pair_kernel<true>, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_bf16_pair_kernel<true, false>, &cfg);
   if (e != cudaSuccess) return e;
   g_pair_clusters[dev] = n + 1;
   return cudaSuccess;
 }
 
 cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                                     void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
-                                     int64_t* launches) {
-  if (p.is_fp8) return cudaErrorNotSupported;
+                                     void* out, const LayoutPtrs& lp, const int32_t* src_row, int max_pair_tiles,
+                                     int n_sms, cudaStream_t s, int64_t* launches) {
+  if (p.is_fp8 || (src_row && !p.swiglu)) return cudaErrorNotSupported;
   int dev = 0;
   cudaError_t e = current_device(&dev);
   if (e != cudaSuccess) return e;
@@ -572,12 +628,17 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& 
   cfg.dynamicSmemBytes = kPairSmemBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   const CUtensorMap& a = reinterpret_cast<const CUtensorMap&>(tm_a);
   const CUtensorMap& b = reinterpret_cast<const CUtensorMap&>(tm_b);
-  if (p.swiglu)
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<true>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
-                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, counter, lp.status);
+  const int32_t* no_rows = nullptr;
+  if (src_row) cfg.blockDim = dim3(kPairThreadsGather, 1, 1);
+  if (src_row)
+    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<true, true>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
+                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, src_row, counter, lp.status);
+  else if (p.swiglu)
+    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<true, false>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
+                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, no_rows, counter, lp.status);
   else
-    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<false>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
-                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, counter, lp.status);
+    e = cudaLaunchKernelEx(&cfg, grouped_gemm_bf16_pair_kernel<false, false>, a, b, num_kb, n_blocks_n, n_group, n_experts, n_out_cols, out_ld,
+                           o, (const int32_t*)lp.tile_prefix, (const int32_t*)lp.counts, (const int32_t*)lp.padded_offsets, no_rows, counter, lp.status);
   *launches += 1;
   return e;
 }

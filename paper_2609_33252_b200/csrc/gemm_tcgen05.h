@@ -23,9 +23,11 @@ cudaError_t launch_gemm_tcgen05(const GemmProblem& p, const GemmTensorMap& tm_a,
 
 // CTA-pair variant (256-row x 256-column tiles, tcgen05 cta_group::2).  box_rows of its weight operand
 // map is gemm_tile_cols()/2.  max_pair_tiles bounds the number of pair tiles (for the grid size).
+// src_row != NULL (GEMM1 only): tm_a describes the caller's token tensor with one-row boxes
+// (make_operand_map with box_rows = 1) and physical row r of the operand is that tensor's row src_row[r].
 cudaError_t launch_gemm_tcgen05_pair(const GemmProblem& p, const GemmTensorMap& tm_a, const GemmTensorMap& tm_b,
-                                     void* out, const LayoutPtrs& lp, int max_pair_tiles, int n_sms, cudaStream_t s,
-                                     int64_t* launches);
+                                     void* out, const LayoutPtrs& lp, const int32_t* src_row, int max_pair_tiles,
+                                     int n_sms, cudaStream_t s, int64_t* launches);
 
 // Block-scaled e4m3 variant.  a_scales [rows, K/128], b_scales [E, N/128, K/128] fp32.  With p.swiglu the output is
 // e4m3 codes [rows, N/2] plus out_scales [rows, N/256]; otherwise bf16 [rows, N].  pair != 0: CTA pairs on 256x256

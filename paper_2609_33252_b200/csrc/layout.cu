@@ -126,7 +126,7 @@ scan_kernel(int n_seg, int E, int32_t* __restrict__ seg_hist /*in: hist, out: ro
 __global__ void __launch_bounds__(kThreads)
 rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t* __restrict__ seg_base,
             int32_t* __restrict__ row_of_pair, int32_t* __restrict__ pair_of_row, int cap_rows,
-            int32_t* __restrict__ status) {
+            int32_t* __restrict__ status, int32_t* __restrict__ src_row /*NULL unless GEMM1 gathers its rows*/) {
   extern __shared__ int32_t sh[];              // [kWarps][E] running row cursor per warp and expert
   pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -175,8 +175,26 @@ rank_kernel(const __grid_constant__ BatchDesc batch, int k, int E, const int32_t
       if (row >= cap_rows) { atomicOr(&status[kStBoundsViolation], 1); row = -1; }
       row_of_pair[p] = row;
       if (row >= 0) pair_of_row[row] = p;
+      if (row >= 0 && src_row) {                 // where the pair's token sits in the caller's token tensor
+        const int t = p / k;
+        int c = 0;
+#pragma unroll 1
+        while (c + 1 < batch.n_chunks && t >= batch.chunk[c + 1].token_base) ++c;
+        src_row[row] = batch.chunk[c].token_offset + (t - batch.chunk[c].token_base);
+      }
     }
   }
+}
+
+// ---- 4'. gather_a plans: no payload moves; only the padding rows' inverse-map entries are marked
+__global__ void __launch_bounds__(128)
+mark_padding_kernel(int E, const int32_t* __restrict__ counts, const int32_t* __restrict__ padded_offsets,
+                    int32_t* __restrict__ pair_of_row, int cap_rows) {
+  pdl_enter();
+  const int e = blockIdx.x;
+  if (e >= E) return;
+  const int r0 = padded_offsets[e] + counts[e], r1 = padded_offsets[e + 1];
+  for (int r = r0 + threadIdx.x; r < r1 && r < cap_rows; r += blockDim.x) pair_of_row[r] = -1;
 }
 
 // ---- 4. payload: one block per token reads its row once and writes it to each local expert's group;
@@ -258,9 +276,16 @@ cudaError_t launch_layout(const BatchDesc& batch, const cep_config& cfg, const L
                    lp.padded_offsets, lp.tile_prefix, lp.sched);
   if (err != cudaSuccess) return err;
   err = launch_pdl(rank_kernel, dim3(n_seg), dim3(kThreads), kWarps * E * sizeof(int32_t), s, 1, batch, k, E,
-                   (const int32_t*)lp.block_base, lp.row_of_pair, lp.pair_of_row, cap_rows, lp.status);
+                   (const int32_t*)lp.block_base, lp.row_of_pair, lp.pair_of_row, cap_rows, lp.status,
+                   cfg.gather_a ? lp.src_row : (int32_t*)nullptr);
   if (err != cudaSuccess) return err;
   if (after_index) { err = cudaEventRecord(after_index, s); if (err != cudaSuccess) return err; }
+  if (cfg.gather_a) {
+    err = launch_pdl(mark_padding_kernel, dim3(E), dim3(128), 0, s, 1, E, (const int32_t*)lp.counts,
+                     (const int32_t*)lp.padded_offsets, lp.pair_of_row, cap_rows);
+    *launches += 4;
+    return err;
+  }
   const bool fp8 = cfg.dtype == CEP_FP8_E4M3_BLOCK128, mx = cfg.dtype == CEP_MXFP4_E4M3;
   const int row_bytes = cfg.hidden * (dtype_is_bytes(cfg.dtype) ? 1 : 2);
   const int n_scale = (fp8 || mx) ? cfg.hidden / kQuantBlock : 0;       // 32-bit scale words per row
@@ -342,7 +367,8 @@ extern "C" int layout_indices_noalloc(const int32_t* topk_ids, int32_t n_tokens,
   hist_kernel<<<(int)n_seg, kThreads, E * sizeof(int32_t), st>>>(batch, top_k, E, n_experts_global, 0, seg_hist, st_words);
   scan_kernel<<<1, 1024, 0, st>>>((int)n_seg, E, seg_hist, counts, offsets, padded_offsets, tile_prefix, scratch + 1600);
   rank_kernel<<<(int)n_seg, kThreads, kWarps * E * sizeof(int32_t), st>>>(batch, top_k, E, seg_hist, row_of_pair,
-                                                                        pair_of_row, pair_of_row_capacity, st_words);
+                                                                        pair_of_row, pair_of_row_capacity, st_words,
+                                                                        (int32_t*)nullptr);
   if (cudaGetLastError() != cudaSuccess) return CEP_ERR_CUDA;
   if (status) {
     // status[0]: an id was outside [0, n_experts_global); status[1]: a row did not fit pair_of_row

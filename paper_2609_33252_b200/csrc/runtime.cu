@@ -63,8 +63,8 @@ bool should_launch(int mode, int64_t pending_pairs, int pending_chunks, int64_t 
 struct Layout {                                   // byte offsets inside the workspace
   size_t status;
   size_t slot0, slot_bytes;
-  size_t counts, offsets, padded, tile_prefix, sched, block_base, row_of_pair, pair_of_row, xp, xp_scales, act,
-      act_scales, y;                              // offsets inside a slot
+  size_t counts, offsets, padded, tile_prefix, sched, block_base, row_of_pair, pair_of_row, src_row, xp, xp_scales,
+      act, act_scales, y;                         // offsets inside a slot
   size_t total;
   int cap_rows, n_seg_max;
   size_t guard;                                   // bytes of poisoned gap after every region (debug_checks)
@@ -87,6 +87,8 @@ int validate(const cep_config* c, const char** why) {
   if (c->n_streams < 1 || c->n_streams > 16) { *why = "n_streams must be in 1..16"; return CEP_ERR_ARG; }
   if (c->threshold_pairs < 0) { *why = "threshold_pairs must be >= 0"; return CEP_ERR_ARG; }
   if (c->gemm_impl < CEP_GEMM_TCGEN05 || c->gemm_impl > CEP_GEMM_TCGEN05_1CTA) { *why = "unknown gemm_impl"; return CEP_ERR_ARG; }
+  if (c->gather_a && (c->dtype != CEP_BF16 || c->gemm_impl != CEP_GEMM_TCGEN05)) {
+    *why = "gather_a is built for bf16 on the CTA-pair tensor-core kernel only"; return CEP_ERR_UNSUPPORTED; }
   return CEP_OK;
 }
 
@@ -117,7 +119,9 @@ Layout make_layout(const cep_config& c) {
   region(L.block_base, (size_t)L.n_seg_max * E * 4, A);
   region(L.row_of_pair, (size_t)max_pairs * 4, A);
   region(L.pair_of_row, (size_t)L.cap_rows * 4, A);
-  region(L.xp, (size_t)L.cap_rows * c.hidden * elt, 1024);
+  // gather_a plans keep no permuted copy of the tokens: GEMM1 reads them where the caller put them
+  region(L.src_row, c.gather_a ? (size_t)L.cap_rows * 4 : 0, A);
+  region(L.xp, c.gather_a ? 0 : (size_t)L.cap_rows * c.hidden * elt, 1024);
   region(L.xp_scales, fp8 ? (size_t)L.cap_rows * (c.hidden / kQuantBlock) * 4 : 0, A);
   region(L.act, (size_t)L.cap_rows * c.inter * elt, 1024);
   region(L.act_scales, fp8 ? (size_t)L.cap_rows * (c.inter / kQuantBlock) * 4 : 0, A);
@@ -176,6 +180,10 @@ struct cep_plan {
   void* s13p; void* s2p;                        // fp8, mxfp4: packed weight scales
   GemmTensorMap tm_b1, tm_b2;
   GemmTensorMap tm_sfb1, tm_sfb2;               // mxfp4: scale atoms of the two weight operands
+  // gather_a: the layer call's token tensor [n_tokens_total, H] as GEMM1's activation operand (one-row boxes);
+  // its base is fixed by the first chunk of the call, every later chunk must be a row slice of the same tensor
+  GemmTensorMap tm_src;
+  const uint8_t* src_base;
   // current layer call
   void* out; const void* addend; int n_tokens_total, n_chunks_expected, n_submitted, tokens_submitted;
   std::vector<char> chunk_seen;
@@ -281,10 +289,11 @@ int launch_invocation(cep_plan* p) {
       const int bn = gemm_tile_cols();
       const long long pair_bound = (m_tiles_bound + groups + 1) / 2;
       const long long t1 = pair_bound * ((g1.N + bn - 1) / bn), t2 = pair_bound * ((g2.N + bn - 1) / bn);
-      CUDA_TRY(p, launch_gemm_tcgen05_pair(g1, sl.tm_a1, p->tm_b1, sl.act, sl.lp, (int)(t1 > (1 << 30) ? (1 << 30) : t1),
+      CUDA_TRY(p, launch_gemm_tcgen05_pair(g1, c.gather_a ? p->tm_src : sl.tm_a1, p->tm_b1, sl.act, sl.lp,
+                                           c.gather_a ? sl.lp.src_row : nullptr, (int)(t1 > (1 << 30) ? (1 << 30) : t1),
                                            p->n_sms, st, &p->launches));
       if (prof) CUDA_TRY(p, cudaEventRecord(iv.mark[1], st));
-      CUDA_TRY(p, launch_gemm_tcgen05_pair(g2, sl.tm_a2, p->tm_b2, sl.y, sl.lp, (int)(t2 > (1 << 30) ? (1 << 30) : t2),
+      CUDA_TRY(p, launch_gemm_tcgen05_pair(g2, sl.tm_a2, p->tm_b2, sl.y, sl.lp, nullptr, (int)(t2 > (1 << 30) ? (1 << 30) : t2),
                                            p->n_sms, st, &p->launches));
     } else {
       const int bn = gemm_tile_cols();
@@ -400,13 +409,14 @@ int moe_plan(const cep_config* cfg, void* workspace, size_t workspace_bytes, cep
     sl.lp.block_base = reinterpret_cast<int32_t*>(b + L.block_base);
     sl.lp.row_of_pair = reinterpret_cast<int32_t*>(b + L.row_of_pair);
     sl.lp.pair_of_row = reinterpret_cast<int32_t*>(b + L.pair_of_row);
+    sl.lp.src_row = cfg->gather_a ? reinterpret_cast<int32_t*>(b + L.src_row) : nullptr;
     sl.lp.status = reinterpret_cast<int32_t*>(p->ws + L.status);
     sl.lp.sched = reinterpret_cast<int32_t*>(b + L.sched);
     sl.xp = b + L.xp; sl.xp_scales = b + L.xp_scales;
     sl.act = b + L.act; sl.act_scales = b + L.act_scales;
     sl.y = b + L.y;
     if (cfg->gemm_impl != CEP_GEMM_SIMT) {
-      int r1 = make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
+      int r1 = cfg->gather_a ? 0 : make_operand_map(&sl.tm_a1, sl.xp, elt, cfg->hidden, L.cap_rows, 0, gemm_tile_rows());
       int r2 = make_operand_map(&sl.tm_a2, sl.act, elt, cfg->inter, L.cap_rows, 0, gemm_tile_rows());
       if (cfg->dtype == CEP_FP8_E4M3_BLOCK128 && !r1 && !r2) {
         r1 = make_store_map(&sl.tm_o1, sl.act, 1, cfg->inter, L.cap_rows);
@@ -500,7 +510,7 @@ int ffn_begin(cep_plan* p, void* out, int32_t n_tokens_total, int32_t n_chunks_e
   CUDA_TRY(p, cudaMemsetAsync(status_dev, 0, kStWords * sizeof(int32_t), s0));
   CUDA_TRY(p, cudaEventRecord(p->begin_evt, s0));
   p->out = out; p->addend = nullptr; p->n_tokens_total = n_tokens_total; p->n_chunks_expected = n_chunks_expected;
-  p->n_submitted = 0; p->tokens_submitted = 0;
+  p->n_submitted = 0; p->tokens_submitted = 0; p->src_base = nullptr;
   p->chunk_seen.assign(n_chunks_expected, 0);
   if (p->call_index >= 0) p->past[p->call_index % kTraceCalls] = p->inv;    // the call that just ended
   p->call_index += 1;
@@ -534,6 +544,17 @@ int ffn_submit_chunk(cep_plan* p, int32_t chunk_id, int32_t token_offset, int32_
   const bool fp8 = dtype_is_bytes(p->cfg.dtype);
   if (fp8 && n_tokens > 0 && !token_scales) return fail(p, CEP_ERR_ARG, "quantised chunk without token_scales");
   if (fp8 && reinterpret_cast<uintptr_t>(token_scales) % 4) return fail(p, CEP_ERR_ARG, "token_scales must be 4-byte aligned");
+  if (p->cfg.gather_a && n_tokens > 0) {
+    // the chunk must be rows token_offset.. of one tensor that holds the whole layer call
+    const uint8_t* base = static_cast<const uint8_t*>(tokens) - (size_t)token_offset * p->cfg.hidden * 2;
+    if (!p->src_base) {
+      if (make_operand_map(&p->tm_src, base, 2, p->cfg.hidden, p->n_tokens_total, 0, 1))
+        return fail(p, CEP_ERR_CUDA, "cuTensorMapEncodeTiled for the token tensor failed");
+      p->src_base = base;
+    } else if (base != p->src_base) {
+      return fail(p, CEP_ERR_UNSUPPORTED, "gather_a: chunk %d is not a row slice of the layer call's token tensor", chunk_id);
+    }
+  }
   const int64_t bound = (int64_t)n_tokens * p->cfg.top_k;
   if (n_local_pairs > bound) return fail(p, CEP_ERR_ARG, "n_local_pairs exceeds n_tokens*top_k");
   const int64_t pairs = n_local_pairs < 0 ? bound : n_local_pairs;

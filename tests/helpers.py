@@ -19,11 +19,11 @@ def chunks_of(inp):
 
 
 def make_layer(cfg, mode=cep.CEP_MODE_SYNC, theta=0, n_streams=2, gemm_impl=cep.CEP_GEMM_TCGEN05, max_chunks=None,
-               debug_checks=0):
+               debug_checks=0, gather_a=0):
     dt = cep.DTYPE_OF[cfg.dtype]
     return cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, max_chunks or max(cfg.n_chunks, 1),
                         dtype=dt, mode=mode, n_streams=n_streams, threshold_pairs=theta, gemm_impl=gemm_impl,
-                        debug_checks=debug_checks)
+                        debug_checks=debug_checks, gather_a=gather_a)
 
 
 def run_layer(inp, layer, order=None, local_pairs=False):

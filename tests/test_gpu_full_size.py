@@ -73,6 +73,16 @@ def test_ep_shard_full_size(name):
     assert n_inv2 > 1
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
     layer.close(); stream.close()
+    if cfg.dtype == "bf16":
+        # the plan without a permuted copy (GEMM1 gathers its rows from the token tensor): same bits, guards intact
+        gathered = make_layer(cfg, mode=cep.CEP_MODE_STREAMFFN, theta=max(1, host.n_local_pairs() // 3), n_streams=2,
+                              debug_checks=1, gather_a=1)
+        gathered.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+        out3, n_inv3 = run_layer(inp, gathered, order=wl.submission_order(host.arrival), local_pairs=True)
+        assert n_inv3 == n_inv2
+        assert cep.cep_debug_check_guards(gathered.plan) == 0
+        assert torch.equal(out.view(torch.int16), out3.view(torch.int16))
+        gathered.close()
 
 
 def test_straggler_config_threshold_sweep_is_bitwise_stable():
