@@ -117,7 +117,7 @@ def sha256_of(path: str) -> str:
         return hashlib.sha256(f.read()).hexdigest()
 
 
-def recorded_traffic(cfg):
+def recorded_traffic(cfg, gather_a=0):
     """GEMM1's measured DRAM bytes per launch for this workload, if a capture of the CURRENT kernel source is on
     record; (None, reason) otherwise."""
     try:
@@ -125,7 +125,7 @@ def recorded_traffic(cfg):
             rec = json.load(f)
     except Exception:
         return None, "no traffic record"
-    ent = rec.get(cfg.name)
+    ent = rec.get(cfg.name + ("+gather_a" if gather_a else ""))
     if ent is None:
         return None, "no capture of this workload on record"
     src = KERNEL_SOURCE[cfg.dtype]
@@ -284,7 +284,7 @@ def main():
     ap.add_argument("--streams", type=int, default=2)
     ap.add_argument("--oracle-tokens", type=int, default=48)
     ap.add_argument("--gemm-impl", type=int, default=0, help="0: CTA-pair tcgen05 (product), 2: one-CTA tcgen05")
-    ap.add_argument("--gather-a", action="store_true",
+    ap.add_argument("--gather-a", type=int, default=0, choices=[0, 1],
                     help="bf16 only: no permuted copy, GEMM1 gathers its rows from the token tensor (cep_config::gather_a); "
                          "applies to the device-resident timing, the end-to-end and arrival sections keep the default")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -332,14 +332,14 @@ def main():
     in_region = args.profile_in_region == 1 or (args.profile_in_region < 0 and work["flops"] >= 2e12)
     layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
                          mode=cep.CEP_MODE_SYNC, n_streams=args.streams, gemm_impl=args.gemm_impl,
-                         profile_kernels=1 if in_region else 0, gather_a=1 if args.gather_a else 0)
+                         profile_kernels=1 if in_region else 0, gather_a=args.gather_a)
     layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     prof_layer = None
     if not in_region:
         # small workloads: a second plan records events between the kernels, run right after the timed region
         prof_layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, cfg.n_chunks, dtype=dt,
                                   mode=cep.CEP_MODE_SYNC, n_streams=1, profile_kernels=1, gemm_impl=args.gemm_impl,
-                                  gather_a=1 if args.gather_a else 0)
+                                  gather_a=args.gather_a)
         prof_layer.load_weights(inp.w_gate, inp.w_up, inp.w_down, inp.s_gate, inp.s_up, inp.s_down)
     torch.cuda.synchronize()
     out = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
@@ -549,9 +549,7 @@ def main():
     #                                                        ratio; the mxf8f6f4 MMA kind (e4m3 x e2m1) runs at the fp8 rate
     burst_tf, sust_tf, nominal_tf = mult * peaks["bf16_tflops"], mult * peaks["bf16_tflops_sustained"], mult * NOMINAL_BF16_TFLOPS
     peak_tf = sust_tf if sustained else burst_tf
-    traffic, traffic_note = recorded_traffic(cfg)
-    if args.gather_a:
-        traffic, traffic_note = None, "no capture of the gathering variant on record"
+    traffic, traffic_note = recorded_traffic(cfg, args.gather_a)
     kernel_sum = sum(med[k_] for k_ in ("layout_ms", "gemm1_ms", "gemm2_ms", "combine_ms"))
     roofline = {"bound": "tensor", "kernel": "grouped GEMM1 (gate/up + SiLU*up%s), CTA-pair tcgen05" %
                           (" + e4m3 re-quantisation" if cfg.dtype != "bf16" else ""),
@@ -592,7 +590,7 @@ def main():
             "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E_local": cfg.E_local,
                        "E_global": cfg.E_global, "top_k": cfg.k, "local_pairs": n_pairs, "chunks": list(cfg.chunks),
                        "mode": "sync (one invocation, all chunks present)", "parallelism": "replicas only",
-                       "gather_a": bool(args.gather_a),
+                       "gather_a": args.gather_a,
                        "l2": "inputs larger than L2 (weights %.2f GB re-read every step)" %
                              (3.0 * cfg.H * cfg.I * {"bf16": 2, "fp8": 1, "mxfp4": 0.5}[cfg.dtype] * cfg.E_local / 1e9)},
             "ffn_tflops": {"value": ffn_tflops, "frac_of_nominal": ffn_tflops / nominal_tf, "nominal_tflops": nominal_tf,
