@@ -123,3 +123,21 @@ def test_refusals():
     assert cep.ffn_status(layer.plan) == 0
     check_close(out, oracle.from_inputs(host), "tiny/gather after a refusal")
     layer.close()
+
+
+def test_library_calibration_runs_on_a_gathering_plan():
+    """The calibration's probe chunks are row slices of one caller buffer, so a gather_a plan profiles itself too."""
+    cfg = wl.MoEConfig("cal", 1, T=2048, H=1024, I=512, E_global=16, E_local=8, k=4, chunks=(2048,))
+    inp = to_device(wl.make_inputs(cfg))
+    layer = cep.MoELayer(cfg.H, cfg.I, cfg.E_global, cfg.E_local, cfg.k, cfg.T, 4, mode=cep.CEP_MODE_ASYNC, n_streams=2,
+                         profile_kernels=1, gather_a=1)
+    layer.load_weights(inp.w_gate, inp.w_up, inp.w_down)
+    ids = torch.empty((cfg.T, cfg.k), dtype=torch.int32, device="cuda")
+    w = torch.empty((cfg.T, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16, device="cuda")
+    points, res = cep.cep_calibrate(layer.plan, 0.9, [32, 128, 512], 2, inp.x, None, ids, w, out)
+    assert [p["rows_per_expert"] for p in points] == [32, 128, 512]
+    assert all(p["ffn_ms"] > 0 for p in points) and res["theta_pairs"] > 0
+    got, _ = run_layer(inp, layer)
+    check_close(got, oracle.from_inputs(wl.make_inputs(cfg)), "gather plan after its calibration")
+    layer.close()
