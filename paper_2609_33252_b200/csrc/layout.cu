@@ -198,7 +198,8 @@ mark_padding_kernel(int E, const int32_t* __restrict__ counts, const int32_t* __
 }
 
 // ---- 4. payload: one block per token reads its row once and writes it to each local expert's group;
-//         E extra blocks zero the padding rows of each group.
+//         the first E blocks zero the padding rows of each group (first, so that the one block that
+//         has up to 127 rows to clear does not run alone at the end).
 template <int kVecPerThread>
 __global__ void __launch_bounds__(kThreads)
 scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int row_bytes, int n_scale,
@@ -208,9 +209,8 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
                     four ue8m0 bytes*/, int sf_atoms /*scale words go to the 512-byte atom order*/, int cap_rows) {
   pdl_enter();
   const int n_vec = row_bytes >> 4;
-  if ((int)blockIdx.x >= batch.n_tokens) {       // padding rows of expert e
-    const int e = blockIdx.x - batch.n_tokens;
-    if (e >= E) return;
+  if ((int)blockIdx.x < E) {                     // padding rows of expert e
+    const int e = blockIdx.x;
     const int r0 = padded_offsets[e] + counts[e], r1 = padded_offsets[e + 1];
     for (int r = r0; r < r1 && r < cap_rows; ++r) {
       uint4* dst = reinterpret_cast<uint4*>(xp + (size_t)r * row_bytes);
@@ -223,7 +223,7 @@ scatter_rows_kernel(const __grid_constant__ BatchDesc batch, int k, int E, int r
     return;
   }
   __shared__ int32_t s_rows[32];
-  const int t = blockIdx.x;
+  const int t = blockIdx.x - E;
   int c = 0;
   while (c + 1 < batch.n_chunks && t >= batch.chunk[c + 1].token_base) ++c;
   const int tl = t - batch.chunk[c].token_base;
